@@ -1,0 +1,357 @@
+#!/usr/bin/env python
+"""Benchmark of the measure -> recover -> execute FFN step.
+
+A step is one pass of the whole path (sketch, recovery, sparse FFN) over one decode batch of a
+synthetic layer.  The default workload is the Llama-2-7B-shaped layer at decode batch 1.  Steps
+rotate over several distinct layers and token batches (more weight bytes than the L2 holds), so
+every step streams its active rows from HBM.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+
+Under torchrun (N > 1) every rank runs the same per-GPU workload on its own tokens (weak scaling,
+no collective on the data path); times are the maximum over ranks.  Prints ONE JSON line.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import torch  # noqa: E402
+
+from gen import workloads as W  # noqa: E402
+
+METRIC = "sparse_ffn_decode_tokens_per_s_per_layer"
+UNIT = "tokens/s"
+GRAPH_STEPS = 64          # steps captured per CUDA graph
+N_TOKEN_BATCHES = 16      # distinct input batches rotated through
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20000)
+    ap.add_argument("--warmup", type=int, default=200)
+    ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--workload", default="l2_7b_b1", choices=["l2_7b_b1", "l2_7b_b64", "l3_8b_stack", "tiny_f32"])
+    ap.add_argument("--layers", type=int, default=0, help="distinct layers rotated through (0 = auto)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    return ap.parse_args()
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return float(p["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML (read-only) while the timed region runs."""
+
+    def __init__(self, index: int, period_s: float = 0.01):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+        self.period = period_s
+
+    def _run(self):
+        nv = self.nv
+        names = {
+            "hw_slowdown": getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8),
+            "hw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40),
+            "sw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20),
+            "sw_power_cap": getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4),
+        }
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                try:
+                    mask = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                except Exception:
+                    mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for k, bit in names.items():
+                    if mask & bit:
+                        self.reasons.add(k)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def __enter__(self):
+        if self.nv is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *exc):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+
+    def summary(self):
+        s = sorted(self.samples)
+        return {"sm_mhz": s[len(s) // 2] if s else None, "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(s)}
+
+
+def algorithmic_bytes(cfg: W.Config, union_groups: float) -> dict:
+    """Bytes the method itself must move per step: active weight blocks (union over the batch,
+    counted once), the sketch matrix, Phi, and the activations in and out."""
+    wbytes = 2 if cfg.w_dtype == "bf16" else 4
+    weights = 3 * union_groups * cfg.group * cfg.d * wbytes
+    sketch = cfg.m * cfg.d * 4 + cfg.m * cfg.G * 4
+    act = 2 * cfg.B * cfg.d * 4
+    return {"weights": weights, "sketch": sketch, "activations": act, "total": weights + sketch + act}
+
+
+def run_ours(args):
+    import paper_2604_14156_b200 as cs
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    cfg = W.CONFIGS[args.workload]
+    wbytes_layer = 3 * cfg.d_ff * cfg.d * (2 if cfg.w_dtype == "bf16" else 4)
+    n_layers = args.layers or (cfg.n_layers if cfg.n_layers > 1 else max(8, int(4e9 // wbytes_layer)))
+    n_layers = min(n_layers, GRAPH_STEPS)
+    K, Wm = args.steps, max(args.warmup, 3)
+
+    plan = cs.Plan(cfg.d, cfg.d_ff, cfg.group, cfg.m, cfg.k, cfg.T,
+                   torch.float32 if cfg.w_dtype == "f32" else torch.bfloat16, cfg.B, cfg.rms_eps)
+    layers_raw, layers = [], []
+    for i in range(n_layers):
+        L = W.make_layer(cfg, i, device=dev)
+        layers_raw.append(L)
+        layers.append(cs.Layer(plan, L.S, L.Phi, L.W_gate, L.W_up, L.Wd_t, L.mu, L.gamma, cfg.rms))
+    # each rank decodes its own tokens (weak scaling): the batch index is offset by the rank
+    xs = torch.stack([W.make_tokens(cfg, layers_raw[0].A, batch=rank * N_TOKEN_BATCHES + j).h
+                      for j in range(N_TOKEN_BATCHES)]).to(dev)
+    x_out = torch.empty_like(xs[0])
+    sup_probe = None
+
+    def step(i):
+        cs.cs_layer_step(plan, layers[i % n_layers], xs[i % N_TOKEN_BATCHES], x_out=x_out, want_aux=False)
+
+    stream = torch.cuda.Stream(device=dev)
+    chunk = min(K, GRAPH_STEPS)
+    with torch.cuda.stream(stream):
+        for i in range(3):
+            step(i)
+        stream.synchronize()
+        before = plan.launches
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            for i in range(chunk):
+                step(i)
+        launches_per_step = (plan.launches - before) / chunk
+
+        def run_steps(n):
+            for _ in range(n // chunk):
+                graph.replay()
+            for i in range(n % chunk):
+                step(i)
+
+        def barrier():
+            if world > 1:
+                import torch.distributed as dist
+                dist.barrier()
+
+        def timed(fn, n):
+            barrier(); torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            fn(n)
+            e1.record(stream)
+            torch.cuda.synchronize(); barrier()
+            ms = e0.elapsed_time(e1)
+            if world > 1:
+                import torch.distributed as dist
+                t = torch.tensor([ms], device=dev, dtype=torch.float64)
+                dist.all_reduce(t, op=dist.ReduceOp.MAX)
+                ms = float(t.item())
+            return ms
+
+        run_steps(Wm)
+        with ClockSampler(local) as clocks:
+            ms_total = timed(run_steps, K)
+
+        # ---- end to end: host buffers in, host result out, through the C boundary
+        hx = torch.stack([x.cpu() for x in xs]).pin_memory()
+        hout = torch.empty_like(hx[0]).pin_memory()
+
+        def step_host(i):
+            cs.cs_layer_step_host(plan, layers[i % n_layers], hx[i % N_TOKEN_BATCHES], hout)
+
+        graph_h = torch.cuda.CUDAGraph()
+        for i in range(3):
+            step_host(i)
+        stream.synchronize()
+        with torch.cuda.graph(graph_h, stream=stream):
+            for i in range(chunk):
+                step_host(i)
+
+        def run_host(n):
+            for _ in range(n // chunk):
+                graph_h.replay()
+            for i in range(n % chunk):
+                step_host(i)
+
+        run_host(min(Wm, chunk))
+        ms_e2e = timed(run_host, K)
+
+        # ---- per-stage device times (separate pass, events around every stage's launches)
+        plan.enable_timing(True)
+        n_prof = min(K, 200)
+        acc = [0.0, 0.0, 0.0, 0.0]
+        for i in range(n_prof + 3):
+            step(i)
+            t = plan.stage_times(stream)
+            if i >= 3:
+                acc = [a + b for a, b in zip(acc, t)]
+        plan.enable_timing(False)
+        stage_ms = [a / n_prof for a in acc]
+        # union of supports of one representative batch (for the algorithmic byte count)
+        _, sup_probe, _, _ = cs.cs_layer_step(plan, layers[0], xs[0])
+        stream.synchronize()
+
+    union = float(len(torch.unique(sup_probe)))
+    tokens = cfg.B * K * world
+    value = tokens / (ms_total * 1e-3)
+    ab = algorithmic_bytes(cfg, union)
+    peak, peak_kind = peaks()
+    exec_ms = stage_ms[2]
+    # the dominant kernel reads the active weights and the hidden state, writes its partial sums
+    kernel_bytes = ab["weights"] + cfg.B * cfg.d * 4 * 2
+    achieved = kernel_bytes / (exec_ms * 1e-3) / 1e9 if exec_ms > 0 else None
+    step_us = ms_total * 1e3 / K
+    mr_us = (stage_ms[0] + stage_ms[1]) * 1e3
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
+        "ms_per_step": ms_total / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic",
+        "config": {"workload": cfg.name, "d": cfg.d, "d_ff": cfg.d_ff, "groups": cfg.G, "group": cfg.group,
+                   "m": cfg.m, "k": cfg.k, "T": cfg.T, "batch": cfg.B, "weights": cfg.w_dtype,
+                   "accumulate": "f32", "layers_rotated": n_layers, "token_batches_rotated": N_TOKEN_BATCHES,
+                   "l2": f"inputs larger than L2: {n_layers} layers x {wbytes_layer / 1e6:.0f} MB rotated",
+                   "cuda_graph_steps": chunk, "parallelism": f"dp{world}" if world > 1 else "single"},
+        "e2e": {"value": tokens / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": cfg.B * cfg.d * 4,
+                "d2h_bytes_per_step": cfg.B * cfg.d * 4},
+        "gpu_launches": int(round(launches_per_step * K)),
+        "clocks": clocks.summary(),
+        "roofline": {"bound": "hbm", "kernel": "ffn_gather_kernel", "achieved": achieved, "peak": peak,
+                     "unit": "GB/s", "frac": (achieved / peak) if achieved else None, "peak_kind": peak_kind,
+                     "frac_of_8tbs_nominal": (achieved / 8000.0) if achieved else None,
+                     "bytes_per_launch": kernel_bytes, "avg_launch_us": exec_ms * 1e3, "traffic": None},
+        "stages_us": {"sketch": stage_ms[0] * 1e3, "recover": stage_ms[1] * 1e3, "exec": stage_ms[2] * 1e3,
+                      "reduce": stage_ms[3] * 1e3, "step_net": step_us,
+                      "measure_recover_per_token": mr_us / cfg.B,
+                      "measure_recover_share_of_step": mr_us / step_us if step_us > 0 else None},
+        "step_hbm": {"algorithmic_bytes": ab["total"], "gbs": ab["total"] / (step_us * 1e-6) / 1e9,
+                     "frac_of_measured_peak": ab["total"] / (step_us * 1e-6) / 1e9 / peak,
+                     "union_groups": union},
+    }
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        out["cpu_baseline"] = cpu_baseline(cfg, [L.to("cpu") for L in layers_raw[:2]], hx, seconds=12.0)
+    if rank == 0:
+        print(json.dumps(out))
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+def cpu_baseline(cfg, cpu_layers, hx, seconds: float):
+    """The fp64 oracle as it stands, on the host cores, on a bounded sample of the same steps."""
+    import oracle
+    n = 0
+    t0 = time.perf_counter()
+    while True:
+        L = cpu_layers[n % len(cpu_layers)]
+        oracle.layer_step(L, hx[n % hx.shape[0]], group=cfg.group, k=cfg.k, T=cfg.T, rms_eps=cfg.rms_eps)
+        n += 1
+        dt = time.perf_counter() - t0
+        if dt >= seconds or n >= 4096:
+            break
+    return {"value": cfg.B * n / dt, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": f"{n} full steps (batch {cfg.B}) of the same workload over {len(cpu_layers)} layers, {dt:.1f} s"}
+
+
+def run_reference(args):
+    """The CPU oracle as the reference arm: K steps on the host cores.  When K full steps would
+    take more than a few minutes, each step runs the full sketch and recovery but the FFN over only
+    the first kk of the k recovered groups, and the FFN time is scaled by k/kk."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import numpy as np
+    import oracle
+    cfg = W.CONFIGS[args.workload]
+    K, Wm = args.steps, max(args.warmup, 1)
+    layers = [W.make_layer(cfg, i) for i in range(2)]
+    xs = [W.make_tokens(cfg, layers[0].A, batch=j).h for j in range(4)]
+
+    def pieces(i, kk):
+        L = layers[i % 2]
+        x = xs[i % 4].double().numpy()
+        t0 = time.perf_counter()
+        n = np.stack([oracle.rmsnorm(x[t], L.gamma, cfg.rms_eps) for t in range(cfg.B)]) if cfg.rms else x
+        y = oracle.sketch(L.S, n)
+        sups = [oracle.iht(L.Phi, y[t], cfg.k, cfg.T, L.mu).support for t in range(cfg.B)]
+        t1 = time.perf_counter()
+        for t in range(cfg.B):
+            oracle.ffn(L.W_gate, L.W_up, L.Wd_t, cfg.group, n[t], sups[t][:kk])
+        t2 = time.perf_counter()
+        return t1 - t0, t2 - t1
+
+    a, b = pieces(0, cfg.k)
+    est = a + b
+    budget = 150.0
+    kk = cfg.k if est * (K + Wm) <= budget else max(1, int(cfg.k * budget / (est * (K + Wm))))
+    for i in range(min(Wm, 3) if kk < cfg.k else Wm):
+        pieces(i, kk)
+    t_sr = t_ffn = 0.0
+    for i in range(K):
+        a, b = pieces(i, kk)
+        t_sr += a; t_ffn += b
+    total = t_sr + t_ffn * (cfg.k / kk)
+    value = cfg.B * K / total
+    sample = (f"{K} full steps" if kk == cfg.k else
+              f"{K} steps, FFN over {kk} of {cfg.k} recovered groups per token, FFN time scaled by {cfg.k}/{kk}")
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": K,
+        "warmup": Wm, "ms_per_step": total / K * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": cfg.name, "d": cfg.d, "d_ff": cfg.d_ff, "groups": cfg.G, "group": cfg.group,
+                   "m": cfg.m, "k": cfg.k, "T": cfg.T, "batch": cfg.B, "weights": cfg.w_dtype},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+if __name__ == "__main__":
+    a = parse_args()
+    if a.impl == "reference":
+        run_reference(a)
+    else:
+        run_ours(a)

@@ -1,0 +1,176 @@
+/*
+ * cs.h -- C boundary of the compressed-sensing-guided sparse FFN step for NVIDIA B200 (sm_100a).
+ *
+ * One transformer SwiGLU FFN layer is executed as the paper's control loop (Sec. 5):
+ *   sensor    y = S n                 a random sketch of the layer's input          (cs_sketch)
+ *   estimator z <- H_k(z + mu Phi^T (y - Phi z)), T times; support = supp(z)         (cs_recover)
+ *   actuator  out = sum over the k recovered channel groups of the SwiGLU FFN        (cs_ffn_exec)
+ * cs_layer_step runs the three for a batch of decode tokens with independent supports;
+ * cs_prompt_support / cs_ffn_exec_shared are the prompt-level variant (Sec. 4) in which one
+ * support is recovered from the mean prompt sketch and shared by every token of the prompt.
+ *
+ * Conventions that hold for every call unless a comment says otherwise
+ *   - Every data pointer is a DEVICE pointer owned by the caller; the library neither frees nor
+ *     keeps it after the call's work has run.  cs_config / cs_layer structs are HOST memory and
+ *     are read before the call returns.
+ *   - Calls only enqueue work on `stream` (a cudaStream_t passed as void*, NULL = default
+ *     stream) and return without synchronising.  A plan must not be used from two streams at
+ *     once: its scratch is shared by all calls.
+ *   - Matrices are dense row-major.  "f32" is IEEE binary32; "bf16" is bfloat16.
+ *   - Errors are return codes.  Arguments are validated on the host before anything is
+ *     launched; on any code other than CS_OK nothing was enqueued.  There is no CPU fallback:
+ *     a shape outside the supported set returns CS_ERR_UNSUPPORTED.
+ *   - Supported shapes: group in {64, 128}; d_ff = G * group with G <= 128; m <= 64;
+ *     1 <= k <= G; d a multiple of 64 and d <= 8192; 1 <= B <= max_tokens.
+ */
+#ifndef CS_H_
+#define CS_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    CS_OK = 0,
+    CS_ERR_NULL = 1,        /* a required pointer is NULL */
+    CS_ERR_SHAPE = 2,       /* sizes inconsistent with the plan (B > max_tokens, n <= 0, ...) */
+    CS_ERR_UNSUPPORTED = 3, /* valid request outside the supported shapes / dtypes */
+    CS_ERR_SUPPORT = 4,     /* device check: a support row is not ascending, distinct and in [0,G) */
+    CS_ERR_NONFINITE = 5,   /* host check: mu or rms_eps is not finite / not positive */
+    CS_ERR_CUDA = 6,        /* a CUDA runtime call failed; see cs_last_cuda_error */
+    CS_ERR_TIMEOUT = 7      /* device check: a bounded wait inside a kernel gave up */
+} cs_status;
+
+typedef enum { CS_F32 = 0, CS_BF16 = 1 } cs_dtype;
+
+/* Shape of one FFN layer and of the recovery problem; fixed for the life of a plan. */
+typedef struct {
+    int32_t d;          /* hidden size */
+    int32_t d_ff;       /* SwiGLU intermediate size = G * group */
+    int32_t group;      /* channels per structured unit ("feed-forward subblock", Sec. 3) */
+    int32_t m;          /* sketch rows (measurement budget m_t, Sec. 3) */
+    int32_t k;          /* active groups per token (sparsity level k_t, Sec. 9) */
+    int32_t T;          /* iterations of the projected iteration (Sec. 8); T = 0 is allowed */
+    int32_t w_dtype;    /* cs_dtype of W_gate / W_up / Wd_t */
+    int32_t max_tokens; /* largest B (and largest prompt length n) any call will pass */
+    float rms_eps;      /* epsilon of the optional RMSNorm */
+} cs_config;
+
+/* Parameters of one layer (device pointers, caller-owned). */
+typedef struct {
+    const float *S;         /* [m, d]    f32  sketch matrix S = Phi * A, precomputed by the caller */
+    const float *Phi;       /* [m, G]    f32  measurement matrix of the recovery problem */
+    const void *W_gate;     /* [d_ff, d] w_dtype */
+    const void *W_up;       /* [d_ff, d] w_dtype */
+    const void *Wd_t;       /* [d_ff, d] w_dtype, W_down TRANSPOSED: row c is column c of W_down */
+    const float *rms_gamma; /* [d] f32 RMSNorm gain, or NULL for no normalisation */
+    float mu;               /* step size of the iteration; 1/||Phi||_2^2 keeps the residual monotone */
+    int32_t add_residual;   /* cs_layer_step: x_out = x + FFN(n) when non-zero, else FFN(n) */
+} cs_layer;
+
+typedef struct cs_plan cs_plan; /* opaque; owns only device scratch sized from cs_config */
+
+/* Validates the configuration and allocates the plan's device scratch on the current device
+ * (the only allocation the library ever makes).  *plan is written only on CS_OK. */
+cs_status cs_plan_create(const cs_config *cfg, cs_plan **plan);
+/* Frees the scratch.  The caller must have synchronised every stream that used the plan. */
+cs_status cs_plan_destroy(cs_plan *plan);
+
+/*
+ * Sensor (Sec. 8, z_t = A_t u_t):  y[t, r] = sum_i S[r, i] * h[t, i].
+ *   S [m,d] f32, h [B,d] f32  ->  y [B,m] f32.  h and y must not overlap.
+ */
+cs_status cs_sketch(cs_plan *plan, const float *S, const float *h, int32_t B, float *y, void *stream);
+
+/*
+ * Estimator (Sec. 7 projection onto the feasible supports, run as the fixed-iteration projected
+ * method of Sec. 8).  For each token independently, from z = 0, T times:
+ *     v = z + mu * Phi^T (y - Phi z);   z = H_k(v)
+ * where H_k keeps the k entries first in the order (|v| descending, group index ascending) and
+ * zeroes the rest.  Always returns exactly k indices (T = 0 gives 0..k-1 and z = 0).
+ *   Phi [m,G] f32, y [B,m] f32  ->  support [B,k] int32 ascending, z [B,k] f32 (z at those
+ *   indices), resid [B] f32 = ||y - Phi z_T||_2 (resid may be NULL; z may be NULL).
+ */
+cs_status cs_recover(cs_plan *plan, const float *Phi, float mu, const float *y, int32_t B,
+                     int32_t *support, float *z, float *resid, void *stream);
+
+/*
+ * Actuator (Sec. 3, execution only on the support), per token t with support s_t:
+ *   a[c]   = silu(W_gate[c,:] . h_t) * (W_up[c,:] . h_t)     for every channel c of a group in s_t
+ *   out[t] = (residual ? residual[t] : 0) + sum_c a[c] * Wd_t[c, :]
+ * silu(x) = x / (1 + exp(-x)).  Products accumulate in f32.
+ *   h [B,d] f32 (the FFN input, already normalised), support [B,k] int32 ascending, distinct,
+ *   in [0,G); residual [B,d] f32 or NULL; out [B,d] f32.  out may alias residual, not h.
+ * layer->S, Phi, rms_gamma, mu and add_residual are ignored.  Small batches run as a gather GEMV
+ * that streams each token's active rows once; large batches bucket tokens by group and run the
+ * active blocks on the tensor cores (activations rounded to bf16 there).
+ */
+cs_status cs_ffn_exec(cs_plan *plan, const cs_layer *layer, const float *h, const int32_t *support,
+                      int32_t B, const float *residual, float *out, void *stream);
+
+/*
+ * One decode step of one layer for B tokens with independent supports (Sec. 5; Sec. 12 online
+ * phase):  n = rms_gamma ? RMSNorm(x) * rms_gamma : x;  y = S n;  (support, z) = recover(y);
+ * x_out = (add_residual ? x : 0) + FFN(n, support).
+ *   x [B,d] f32 -> x_out [B,d] f32 (x_out may alias x).  support_out [B,k], z_out [B,k],
+ *   resid_out [B] may each be NULL.
+ */
+cs_status cs_layer_step(cs_plan *plan, const cs_layer *layer, const float *x, int32_t B, float *x_out,
+                        int32_t *support_out, float *z_out, float *resid_out, void *stream);
+
+/*
+ * Prompt-level support (Sec. 4): one support for the whole prompt from the mean prompt sketch,
+ *   ybar = (1/n) sum_i S h_i  (computed as S applied to the mean hidden state, equal by linearity),
+ * followed by the recovery of cs_recover on ybar.
+ *   H [n,d] bf16  ->  support [k] int32 ascending, z [k] f32 (may be NULL), resid [1] (may be NULL).
+ */
+cs_status cs_prompt_support(cs_plan *plan, const float *S, const float *Phi, float mu, const void *H,
+                            int32_t n, int32_t *support, float *z, float *resid, void *stream);
+
+/*
+ * FFN of every prompt token over ONE shared support (Sec. 4), as grouped dense GEMMs over the k
+ * active row blocks on the tensor cores: bf16 operands, f32 accumulation, the intermediate
+ * activation rounded to bf16 between the two GEMMs.
+ *   H [n,d] bf16, support [k] int32 (device) -> out [n,d] bf16.  Requires w_dtype = CS_BF16,
+ *   group = 128.  out must not overlap H.
+ */
+cs_status cs_ffn_exec_shared(cs_plan *plan, const cs_layer *layer, const void *H, int32_t n,
+                             const int32_t *support, void *out, void *stream);
+
+/*
+ * cs_layer_step for callers whose activations live in HOST memory (ideally pinned): copies
+ * x_host [B,d] f32 to plan scratch, runs the step, copies x_out [B,d] f32 (and, if not NULL,
+ * the supports [B,k] int32) back, all enqueued on `stream`.  The host buffers must stay valid
+ * until the stream has been synchronised.  Per step it moves 4*B*d bytes each way.
+ */
+cs_status cs_layer_step_host(cs_plan *plan, const cs_layer *layer, const float *x_host, int32_t B,
+                             float *x_out_host, int32_t *support_host, void *stream);
+
+/*
+ * Stage timing (the paper asks for sensing / recovery overhead to be reported apart from the
+ * sparse kernel itself, Sec. 15 metric suite).  While enabled, every launch of a stage is bracketed
+ * by CUDA events on the call's stream.  cs_plan_stage_times synchronises `stream` and returns the
+ * device time in milliseconds of each stage's kernels in the most recent call that ran it.
+ */
+enum { CS_STAGE_SKETCH = 0, CS_STAGE_RECOVER = 1, CS_STAGE_EXEC = 2, CS_STAGE_REDUCE = 3, CS_STAGE_COUNT = 4 };
+cs_status cs_plan_enable_timing(cs_plan *plan, int32_t on);
+cs_status cs_plan_stage_times(cs_plan *plan, void *stream, float ms[CS_STAGE_COUNT]);
+
+/* Reads (and clears) the plan's device status word, synchronising `stream` first: CS_OK, or the
+ * first CS_ERR_SUPPORT / CS_ERR_TIMEOUT a kernel recorded since the last read. */
+cs_status cs_last_device_status(cs_plan *plan, void *stream, int32_t *code);
+
+/* Number of kernels the library has launched through this plan since it was created. */
+int64_t cs_launch_count(const cs_plan *plan);
+
+/* Text of the last CUDA runtime error seen by this plan ("" if none); valid until the next call. */
+const char *cs_last_cuda_error(const cs_plan *plan);
+
+const char *cs_status_string(cs_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CS_H_ */

@@ -1,0 +1,264 @@
+"""ctypes binding of libcs_b200.so (argument marshalling only)."""
+from __future__ import annotations
+
+import ctypes
+import os
+import re
+from typing import Optional
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_PKG, "libcs_b200.so")
+_HEADER = os.path.join(os.path.dirname(_PKG), "include", "cs.h")
+
+CS_F32, CS_BF16 = 0, 1
+_STATUS_NAMES = {0: "CS_OK", 1: "CS_ERR_NULL", 2: "CS_ERR_SHAPE", 3: "CS_ERR_UNSUPPORTED",
+                 4: "CS_ERR_SUPPORT", 5: "CS_ERR_NONFINITE", 6: "CS_ERR_CUDA", 7: "CS_ERR_TIMEOUT"}
+
+
+class CSError(RuntimeError):
+    def __init__(self, code: int, where: str, detail: str = ""):
+        self.code = code
+        super().__init__(f"{where}: {_STATUS_NAMES.get(code, code)}" + (f" ({detail})" if detail else ""))
+
+
+class _Config(ctypes.Structure):
+    _fields_ = [("d", ctypes.c_int32), ("d_ff", ctypes.c_int32), ("group", ctypes.c_int32),
+                ("m", ctypes.c_int32), ("k", ctypes.c_int32), ("T", ctypes.c_int32),
+                ("w_dtype", ctypes.c_int32), ("max_tokens", ctypes.c_int32), ("rms_eps", ctypes.c_float)]
+
+
+class _Layer(ctypes.Structure):
+    _fields_ = [("S", ctypes.c_void_p), ("Phi", ctypes.c_void_p), ("W_gate", ctypes.c_void_p),
+                ("W_up", ctypes.c_void_p), ("Wd_t", ctypes.c_void_p), ("rms_gamma", ctypes.c_void_p),
+                ("mu", ctypes.c_float), ("add_residual", ctypes.c_int32)]
+
+
+def library_path() -> str:
+    return _LIB_PATH
+
+
+def exported_symbols():
+    """Names of the functions include/cs.h declares (used by the load test)."""
+    text = open(_HEADER).read()
+    return sorted(set(re.findall(r"\b(cs_[a-z_]+)\s*\(", text)))
+
+
+_lib = None
+
+
+def load_library():
+    """Load libcs_b200.so; there is no fallback if it has not been built."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(_LIB_PATH):
+        raise ImportError(f"{_LIB_PATH} is missing: build it with `python -m paper_2604_14156_b200.build` "
+                          "(there is no CPU path)")
+    lib = ctypes.CDLL(_LIB_PATH)
+    vp, i32, f32 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_float
+    lib.cs_plan_create.argtypes = [ctypes.POINTER(_Config), ctypes.POINTER(vp)]
+    lib.cs_plan_destroy.argtypes = [vp]
+    lib.cs_sketch.argtypes = [vp, vp, vp, i32, vp, vp]
+    lib.cs_recover.argtypes = [vp, vp, f32, vp, i32, vp, vp, vp, vp]
+    lib.cs_ffn_exec.argtypes = [vp, ctypes.POINTER(_Layer), vp, vp, i32, vp, vp, vp]
+    lib.cs_layer_step.argtypes = [vp, ctypes.POINTER(_Layer), vp, i32, vp, vp, vp, vp, vp]
+    lib.cs_prompt_support.argtypes = [vp, vp, vp, f32, vp, i32, vp, vp, vp, vp]
+    lib.cs_ffn_exec_shared.argtypes = [vp, ctypes.POINTER(_Layer), vp, i32, vp, vp, vp]
+    lib.cs_layer_step_host.argtypes = [vp, ctypes.POINTER(_Layer), vp, i32, vp, vp, vp]
+    lib.cs_plan_enable_timing.argtypes = [vp, i32]
+    lib.cs_plan_stage_times.argtypes = [vp, vp, ctypes.POINTER(f32 * 4)]
+    lib.cs_last_device_status.argtypes = [vp, vp, ctypes.POINTER(i32)]
+    lib.cs_launch_count.argtypes = [vp]
+    lib.cs_launch_count.restype = ctypes.c_int64
+    lib.cs_last_cuda_error.argtypes = [vp]
+    lib.cs_last_cuda_error.restype = ctypes.c_char_p
+    lib.cs_status_string.argtypes = [ctypes.c_int]
+    lib.cs_status_string.restype = ctypes.c_char_p
+    for name in ("cs_plan_create", "cs_plan_destroy", "cs_sketch", "cs_recover", "cs_ffn_exec",
+                 "cs_layer_step", "cs_prompt_support", "cs_ffn_exec_shared", "cs_last_device_status",
+                 "cs_layer_step_host", "cs_plan_enable_timing", "cs_plan_stage_times"):
+        getattr(lib, name).restype = ctypes.c_int
+    _lib = lib
+    return lib
+
+
+def _ptr(t: Optional[torch.Tensor], dtype: torch.dtype, name: str, shape=None) -> Optional[int]:
+    if t is None:
+        return None
+    if not t.is_cuda:
+        raise TypeError(f"{name} must be a CUDA tensor (the library has no CPU path)")
+    if t.dtype != dtype:
+        raise TypeError(f"{name} must be {dtype}, got {t.dtype}")
+    if not t.is_contiguous():
+        raise ValueError(f"{name} must be contiguous")
+    if shape is not None and tuple(t.shape) != tuple(shape):
+        raise ValueError(f"{name} must have shape {tuple(shape)}, got {tuple(t.shape)}")
+    return t.data_ptr()
+
+
+def _stream(stream) -> int:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return stream.cuda_stream
+
+
+class Plan:
+    """Owns a cs_plan (device scratch sized for one layer shape)."""
+
+    def __init__(self, d: int, d_ff: int, group: int, m: int, k: int, T: int, w_dtype: torch.dtype,
+                 max_tokens: int, rms_eps: float = 1e-5):
+        self.lib = load_library()
+        self.d, self.d_ff, self.group, self.m, self.k, self.T = d, d_ff, group, m, k, T
+        self.G = d_ff // group if group > 0 else 0
+        self.w_dtype = w_dtype
+        self.max_tokens = max_tokens
+        code = {torch.float32: CS_F32, torch.bfloat16: CS_BF16}.get(w_dtype, -1)
+        cfg = _Config(d, d_ff, group, m, k, T, code, max_tokens, rms_eps)
+        handle = ctypes.c_void_p()
+        st = self.lib.cs_plan_create(ctypes.byref(cfg), ctypes.byref(handle))
+        self.handle = None
+        if st != 0:
+            raise CSError(st, "cs_plan_create")
+        self.handle = handle
+
+    def check(self, st: int, where: str):
+        if st != 0:
+            detail = self.lib.cs_last_cuda_error(self.handle).decode() if st == 6 else ""
+            raise CSError(st, where, detail)
+
+    def device_status(self, stream=None) -> int:
+        code = ctypes.c_int32(0)
+        self.check(self.lib.cs_last_device_status(self.handle, _stream(stream), ctypes.byref(code)),
+                   "cs_last_device_status")
+        return code.value
+
+    def enable_timing(self, on: bool = True):
+        self.check(self.lib.cs_plan_enable_timing(self.handle, int(on)), "cs_plan_enable_timing")
+
+    def stage_times(self, stream=None):
+        """Milliseconds of (sketch, recover, exec, reduce) in the most recent call."""
+        ms = (ctypes.c_float * 4)()
+        self.check(self.lib.cs_plan_stage_times(self.handle, _stream(stream), ctypes.byref(ms)),
+                   "cs_plan_stage_times")
+        return tuple(ms)
+
+    @property
+    def launches(self) -> int:
+        return int(self.lib.cs_launch_count(self.handle))
+
+    def close(self):
+        if self.handle is not None:
+            self.lib.cs_plan_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+class Layer:
+    """Device tensors of one layer; keeps them alive and exposes the C struct."""
+
+    def __init__(self, plan: Plan, S, Phi, W_gate, W_up, Wd_t, mu: float, rms_gamma=None,
+                 add_residual: bool = False):
+        G = plan.G
+        self.tensors = (S, Phi, W_gate, W_up, Wd_t, rms_gamma)
+        self.c = _Layer(
+            _ptr(S, torch.float32, "S", (plan.m, plan.d)), _ptr(Phi, torch.float32, "Phi", (plan.m, G)),
+            _ptr(W_gate, plan.w_dtype, "W_gate", (plan.d_ff, plan.d)),
+            _ptr(W_up, plan.w_dtype, "W_up", (plan.d_ff, plan.d)),
+            _ptr(Wd_t, plan.w_dtype, "Wd_t", (plan.d_ff, plan.d)),
+            _ptr(rms_gamma, torch.float32, "rms_gamma", (plan.d,)), float(mu), int(bool(add_residual)))
+        self.mu = float(mu)
+        self.S, self.Phi = S, Phi
+
+
+def cs_sketch(plan: Plan, S, h, y=None, stream=None):
+    B = h.shape[0]
+    y = torch.empty((B, plan.m), dtype=torch.float32, device=h.device) if y is None else y
+    plan.check(plan.lib.cs_sketch(plan.handle, _ptr(S, torch.float32, "S", (plan.m, plan.d)),
+                                  _ptr(h, torch.float32, "h", (B, plan.d)), B,
+                                  _ptr(y, torch.float32, "y", (B, plan.m)), _stream(stream)), "cs_sketch")
+    return y
+
+
+def cs_recover(plan: Plan, Phi, mu: float, y, stream=None):
+    B = y.shape[0]
+    dev = y.device
+    support = torch.empty((B, plan.k), dtype=torch.int32, device=dev)
+    z = torch.empty((B, plan.k), dtype=torch.float32, device=dev)
+    resid = torch.empty((B,), dtype=torch.float32, device=dev)
+    plan.check(plan.lib.cs_recover(plan.handle, _ptr(Phi, torch.float32, "Phi", (plan.m, plan.G)), float(mu),
+                                   _ptr(y, torch.float32, "y", (B, plan.m)), B, support.data_ptr(),
+                                   z.data_ptr(), resid.data_ptr(), _stream(stream)), "cs_recover")
+    return support, z, resid
+
+
+def cs_ffn_exec(plan: Plan, layer: Layer, h, support, residual=None, out=None, stream=None):
+    B = h.shape[0]
+    out = torch.empty((B, plan.d), dtype=torch.float32, device=h.device) if out is None else out
+    plan.check(plan.lib.cs_ffn_exec(plan.handle, ctypes.byref(layer.c), _ptr(h, torch.float32, "h", (B, plan.d)),
+                                    _ptr(support, torch.int32, "support", (B, plan.k)), B,
+                                    _ptr(residual, torch.float32, "residual", (B, plan.d)),
+                                    _ptr(out, torch.float32, "out", (B, plan.d)), _stream(stream)), "cs_ffn_exec")
+    return out
+
+
+def cs_layer_step(plan: Plan, layer: Layer, x, x_out=None, want_aux: bool = True, stream=None):
+    """Returns (x_out, support, z, resid); the last three are None when want_aux is False."""
+    B = x.shape[0]
+    dev = x.device
+    x_out = torch.empty_like(x) if x_out is None else x_out
+    support = z = resid = None
+    if want_aux:
+        support = torch.empty((B, plan.k), dtype=torch.int32, device=dev)
+        z = torch.empty((B, plan.k), dtype=torch.float32, device=dev)
+        resid = torch.empty((B,), dtype=torch.float32, device=dev)
+    plan.check(plan.lib.cs_layer_step(plan.handle, ctypes.byref(layer.c), _ptr(x, torch.float32, "x", (B, plan.d)), B,
+                                      _ptr(x_out, torch.float32, "x_out", (B, plan.d)),
+                                      None if support is None else support.data_ptr(),
+                                      None if z is None else z.data_ptr(),
+                                      None if resid is None else resid.data_ptr(), _stream(stream)),
+               "cs_layer_step")
+    return x_out, support, z, resid
+
+
+def cs_layer_step_host(plan: Plan, layer: Layer, x_host, x_out_host, support_host=None, stream=None):
+    """x_host / x_out_host: CPU float32 tensors [B, d] (pinned for asynchronous copies)."""
+    B = x_host.shape[0]
+    for t, name in ((x_host, "x_host"), (x_out_host, "x_out_host")):
+        if t.is_cuda or t.dtype != torch.float32 or not t.is_contiguous() or tuple(t.shape) != (B, plan.d):
+            raise TypeError(f"{name} must be a contiguous CPU float32 tensor of shape ({B}, {plan.d})")
+    plan.check(plan.lib.cs_layer_step_host(plan.handle, ctypes.byref(layer.c), x_host.data_ptr(), B,
+                                           x_out_host.data_ptr(),
+                                           None if support_host is None else support_host.data_ptr(),
+                                           _stream(stream)), "cs_layer_step_host")
+    return x_out_host
+
+
+def cs_prompt_support(plan: Plan, S, Phi, mu: float, H, stream=None):
+    n = H.shape[0]
+    dev = H.device
+    support = torch.empty((plan.k,), dtype=torch.int32, device=dev)
+    z = torch.empty((plan.k,), dtype=torch.float32, device=dev)
+    resid = torch.empty((1,), dtype=torch.float32, device=dev)
+    plan.check(plan.lib.cs_prompt_support(plan.handle, _ptr(S, torch.float32, "S", (plan.m, plan.d)),
+                                          _ptr(Phi, torch.float32, "Phi", (plan.m, plan.G)), float(mu),
+                                          _ptr(H, torch.bfloat16, "H", (n, plan.d)), n, support.data_ptr(),
+                                          z.data_ptr(), resid.data_ptr(), _stream(stream)), "cs_prompt_support")
+    return support, z, resid
+
+
+def cs_ffn_exec_shared(plan: Plan, layer: Layer, H, support, out=None, stream=None):
+    n = H.shape[0]
+    out = torch.empty_like(H) if out is None else out
+    plan.check(plan.lib.cs_ffn_exec_shared(plan.handle, ctypes.byref(layer.c),
+                                           _ptr(H, torch.bfloat16, "H", (n, plan.d)), n,
+                                           _ptr(support, torch.int32, "support", (plan.k,)),
+                                           _ptr(out, torch.bfloat16, "out", (n, plan.d)), _stream(stream)),
+               "cs_ffn_exec_shared")
+    return out

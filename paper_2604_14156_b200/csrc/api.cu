@@ -1,0 +1,237 @@
+// The C boundary: plan life cycle, host-side validation and dispatch.  See include/cs.h.
+#include <math.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <new>
+
+#include "cs_internal.cuh"
+
+namespace cs {
+
+cs_status record_cuda(cs_plan *plan, cudaError_t e, const char *what) {
+    if (plan != nullptr)
+        snprintf(plan->cuda_error, sizeof plan->cuda_error, "%s: %s", what, cudaGetErrorString(e));
+    return CS_ERR_CUDA;
+}
+
+static cs_status check_config(const cs_config *c) {
+    if (c->d <= 0 || c->d_ff <= 0 || c->group <= 0 || c->m <= 0 || c->k <= 0 || c->T < 0 || c->max_tokens <= 0)
+        return CS_ERR_SHAPE;
+    if (c->d_ff % c->group != 0) return CS_ERR_SHAPE;
+    const int G = c->d_ff / c->group;
+    if (c->k > G) return CS_ERR_SHAPE;
+    if (!(c->rms_eps > 0.f) || !isfinite(c->rms_eps)) return CS_ERR_NONFINITE;
+    if (c->group != 64 && c->group != 128) return CS_ERR_UNSUPPORTED;
+    if (G > kMaxG || c->m > kMaxM || c->d > kMaxD || c->d % 64 != 0) return CS_ERR_UNSUPPORTED;
+    if (c->w_dtype != CS_F32 && c->w_dtype != CS_BF16) return CS_ERR_UNSUPPORTED;
+    return CS_OK;
+}
+
+static bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+}  // namespace cs
+
+using namespace cs;
+
+extern "C" {
+
+cs_status cs_plan_create(const cs_config *cfg, cs_plan **out) {
+    if (cfg == nullptr || out == nullptr) return CS_ERR_NULL;
+    cs_status s = check_config(cfg);
+    if (s != CS_OK) return s;
+    cs_plan *p = new (std::nothrow) cs_plan();
+    if (p == nullptr) return CS_ERR_CUDA;
+    memset(p, 0, sizeof *p);
+    p->cfg = *cfg;
+    p->G = cfg->d_ff / cfg->group;
+    cudaError_t e = cudaGetDevice(&p->device);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&p->sm_count, cudaDevAttrMultiProcessorCount, p->device);
+    const size_t nt = (size_t)cfg->max_tokens;
+    p->nx_max = max(p->sm_count, (cfg->k * cfg->group + kGatherMaxRows - 1) / kGatherMaxRows);
+    p->mean_row_blocks = 32;
+    auto alloc = [&](void **ptr, size_t bytes) {
+        if (e == cudaSuccess) e = cudaMalloc(ptr, bytes);
+    };
+    alloc((void **)&p->n_buf, nt * cfg->d * sizeof(float));
+    alloc((void **)&p->y_buf, nt * cfg->m * sizeof(float));
+    alloc((void **)&p->sup_buf, nt * cfg->k * sizeof(int32_t));
+    alloc((void **)&p->z_buf, nt * cfg->k * sizeof(float));
+    alloc((void **)&p->resid_buf, nt * sizeof(float));
+    alloc((void **)&p->partial, (size_t)kGatherMaxTokens * p->nx_max * cfg->d * sizeof(float));
+    alloc((void **)&p->hbar, (size_t)cfg->d * sizeof(float));
+    alloc((void **)&p->colsum, (size_t)p->mean_row_blocks * cfg->d * sizeof(float));
+    alloc((void **)&p->status, sizeof(DeviceStatus));
+    alloc((void **)&p->x_host_in, nt * cfg->d * sizeof(float));
+    alloc((void **)&p->x_host_out, nt * cfg->d * sizeof(float));
+    for (int i = 0; i < 2 * CS_STAGE_COUNT; ++i)
+        if (e == cudaSuccess) e = cudaEventCreate(&p->ev[i]);
+    if (e == cudaSuccess) e = cudaMemset(p->status, 0, sizeof(DeviceStatus));
+    if (e != cudaSuccess) {
+        cs_plan_destroy(p);
+        return CS_ERR_CUDA;
+    }
+    *out = p;
+    return CS_OK;
+}
+
+cs_status cs_plan_destroy(cs_plan *p) {
+    if (p == nullptr) return CS_ERR_NULL;
+    cudaFree(p->n_buf); cudaFree(p->y_buf); cudaFree(p->sup_buf); cudaFree(p->z_buf);
+    cudaFree(p->resid_buf); cudaFree(p->partial); cudaFree(p->hbar); cudaFree(p->colsum);
+    cudaFree(p->status); cudaFree(p->x_host_in); cudaFree(p->x_host_out);
+    for (int i = 0; i < 2 * CS_STAGE_COUNT; ++i)
+        if (p->ev[i] != nullptr) cudaEventDestroy(p->ev[i]);
+    delete p;
+    return CS_OK;
+}
+
+cs_status cs_sketch(cs_plan *plan, const float *S, const float *h, int32_t B, float *y, void *stream) {
+    if (plan == nullptr || S == nullptr || h == nullptr || y == nullptr) return CS_ERR_NULL;
+    if (B <= 0 || B > plan->cfg.max_tokens) return CS_ERR_SHAPE;
+    if (!aligned16(S) || !aligned16(h)) return CS_ERR_UNSUPPORTED;
+    return launch_sketch(plan, S, h, nullptr, B, y, nullptr, static_cast<cudaStream_t>(stream));
+}
+
+cs_status cs_recover(cs_plan *plan, const float *Phi, float mu, const float *y, int32_t B,
+                     int32_t *support, float *z, float *resid, void *stream) {
+    if (plan == nullptr || Phi == nullptr || y == nullptr || support == nullptr) return CS_ERR_NULL;
+    if (B <= 0 || B > plan->cfg.max_tokens) return CS_ERR_SHAPE;
+    if (!isfinite(mu) || !(mu > 0.f)) return CS_ERR_NONFINITE;
+    return launch_recover(plan, Phi, mu, y, B, support, z, resid, static_cast<cudaStream_t>(stream));
+}
+
+static cs_status check_weights(const cs_layer *L) {
+    if (L == nullptr || L->W_gate == nullptr || L->W_up == nullptr || L->Wd_t == nullptr) return CS_ERR_NULL;
+    if (!aligned16(L->W_gate) || !aligned16(L->W_up) || !aligned16(L->Wd_t)) return CS_ERR_UNSUPPORTED;
+    return CS_OK;
+}
+
+cs_status cs_ffn_exec(cs_plan *plan, const cs_layer *layer, const float *h, const int32_t *support,
+                      int32_t B, const float *residual, float *out, void *stream) {
+    if (plan == nullptr || h == nullptr || support == nullptr || out == nullptr) return CS_ERR_NULL;
+    cs_status s = check_weights(layer);
+    if (s != CS_OK) return s;
+    if (B <= 0 || B > plan->cfg.max_tokens) return CS_ERR_SHAPE;
+    if (!aligned16(h) || !aligned16(out) || (residual != nullptr && !aligned16(residual))) return CS_ERR_UNSUPPORTED;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    s = launch_check_support(plan, support, B, st);
+    if (s != CS_OK) return s;
+    return launch_ffn_gather(plan, layer, h, support, B, residual, out, st);
+}
+
+cs_status cs_layer_step(cs_plan *plan, const cs_layer *layer, const float *x, int32_t B, float *x_out,
+                        int32_t *support_out, float *z_out, float *resid_out, void *stream) {
+    if (plan == nullptr || x == nullptr || x_out == nullptr) return CS_ERR_NULL;
+    cs_status s = check_weights(layer);
+    if (s != CS_OK) return s;
+    if (layer->S == nullptr || layer->Phi == nullptr) return CS_ERR_NULL;
+    if (B <= 0 || B > plan->cfg.max_tokens) return CS_ERR_SHAPE;
+    if (!isfinite(layer->mu) || !(layer->mu > 0.f)) return CS_ERR_NONFINITE;
+    if (!aligned16(x) || !aligned16(x_out) || !aligned16(layer->S) ||
+        (layer->rms_gamma != nullptr && !aligned16(layer->rms_gamma)))
+        return CS_ERR_UNSUPPORTED;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const bool norm = layer->rms_gamma != nullptr;
+    const float *n = norm ? plan->n_buf : x;
+    int32_t *sup = support_out != nullptr ? support_out : plan->sup_buf;
+    s = launch_sketch(plan, layer->S, x, layer->rms_gamma, B, plan->y_buf, norm ? plan->n_buf : nullptr, st);
+    if (s != CS_OK) return s;
+    s = launch_recover(plan, layer->Phi, layer->mu, plan->y_buf, B, sup, z_out, resid_out, st);
+    if (s != CS_OK) return s;
+    // supports produced by cs_recover are valid by construction: no device check here
+    return launch_ffn_gather(plan, layer, n, sup, B, layer->add_residual ? x : nullptr, x_out, st);
+}
+
+cs_status cs_layer_step_host(cs_plan *plan, const cs_layer *layer, const float *x_host, int32_t B,
+                             float *x_out_host, int32_t *support_host, void *stream) {
+    if (plan == nullptr || x_host == nullptr || x_out_host == nullptr) return CS_ERR_NULL;
+    if (B <= 0 || B > plan->cfg.max_tokens) return CS_ERR_SHAPE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t bytes = (size_t)B * plan->cfg.d * sizeof(float);
+    // validate before the first copy so that nothing is enqueued on an error
+    cs_status s = check_weights(layer);
+    if (s != CS_OK) return s;
+    if (layer->S == nullptr || layer->Phi == nullptr) return CS_ERR_NULL;
+    if (!isfinite(layer->mu) || !(layer->mu > 0.f)) return CS_ERR_NONFINITE;
+    CS_CUDA_TRY(plan, cudaMemcpyAsync(plan->x_host_in, x_host, bytes, cudaMemcpyHostToDevice, st));
+    s = cs_layer_step(plan, layer, plan->x_host_in, B, plan->x_host_out, plan->sup_buf, nullptr, nullptr, stream);
+    if (s != CS_OK) return s;
+    CS_CUDA_TRY(plan, cudaMemcpyAsync(x_out_host, plan->x_host_out, bytes, cudaMemcpyDeviceToHost, st));
+    if (support_host != nullptr)
+        CS_CUDA_TRY(plan, cudaMemcpyAsync(support_host, plan->sup_buf, (size_t)B * plan->cfg.k * sizeof(int32_t),
+                                          cudaMemcpyDeviceToHost, st));
+    return CS_OK;
+}
+
+cs_status cs_plan_enable_timing(cs_plan *plan, int32_t on) {
+    if (plan == nullptr) return CS_ERR_NULL;
+    plan->timing = on != 0;
+    for (int i = 0; i < CS_STAGE_COUNT; ++i) plan->stage_seen[i] = 0;
+    return CS_OK;
+}
+
+cs_status cs_plan_stage_times(cs_plan *plan, void *stream, float ms[CS_STAGE_COUNT]) {
+    if (plan == nullptr || ms == nullptr) return CS_ERR_NULL;
+    CS_CUDA_TRY(plan, cudaStreamSynchronize(static_cast<cudaStream_t>(stream)));
+    for (int i = 0; i < CS_STAGE_COUNT; ++i) {
+        ms[i] = 0.f;
+        if (plan->stage_seen[i]) CS_CUDA_TRY(plan, cudaEventElapsedTime(&ms[i], plan->ev[2 * i], plan->ev[2 * i + 1]));
+    }
+    return CS_OK;
+}
+
+cs_status cs_prompt_support(cs_plan *plan, const float *S, const float *Phi, float mu, const void *H,
+                            int32_t n, int32_t *support, float *z, float *resid, void *stream) {
+    if (plan == nullptr || S == nullptr || Phi == nullptr || H == nullptr || support == nullptr) return CS_ERR_NULL;
+    if (n <= 0 || n > plan->cfg.max_tokens) return CS_ERR_SHAPE;
+    if (!isfinite(mu) || !(mu > 0.f)) return CS_ERR_NONFINITE;
+    if (!aligned16(S) || !aligned16(H)) return CS_ERR_UNSUPPORTED;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cs_status s = launch_prompt_mean(plan, H, n, plan->hbar, st);
+    if (s != CS_OK) return s;
+    s = launch_sketch(plan, S, plan->hbar, nullptr, 1, plan->y_buf, nullptr, st);
+    if (s != CS_OK) return s;
+    return launch_recover(plan, Phi, mu, plan->y_buf, 1, support, z, resid, st);
+}
+
+cs_status cs_ffn_exec_shared(cs_plan *plan, const cs_layer *layer, const void *H, int32_t n,
+                             const int32_t *support, void *out, void *stream) {
+    if (plan == nullptr || H == nullptr || support == nullptr || out == nullptr) return CS_ERR_NULL;
+    cs_status s = check_weights(layer);
+    if (s != CS_OK) return s;
+    if (n <= 0 || n > plan->cfg.max_tokens) return CS_ERR_SHAPE;
+    (void)stream;
+    return CS_ERR_UNSUPPORTED;
+}
+
+cs_status cs_last_device_status(cs_plan *plan, void *stream, int32_t *code) {
+    if (plan == nullptr || code == nullptr) return CS_ERR_NULL;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    DeviceStatus hs;
+    CS_CUDA_TRY(plan, cudaMemcpyAsync(&hs, plan->status, sizeof hs, cudaMemcpyDeviceToHost, st));
+    CS_CUDA_TRY(plan, cudaMemsetAsync(plan->status, 0, sizeof hs, st));
+    CS_CUDA_TRY(plan, cudaStreamSynchronize(st));
+    *code = hs.code;
+    return CS_OK;
+}
+
+int64_t cs_launch_count(const cs_plan *plan) { return plan != nullptr ? plan->launches : 0; }
+
+const char *cs_last_cuda_error(const cs_plan *plan) { return plan != nullptr ? plan->cuda_error : ""; }
+
+const char *cs_status_string(cs_status s) {
+    switch (s) {
+        case CS_OK: return "ok";
+        case CS_ERR_NULL: return "null pointer";
+        case CS_ERR_SHAPE: return "inconsistent shape";
+        case CS_ERR_UNSUPPORTED: return "unsupported shape, dtype or alignment";
+        case CS_ERR_SUPPORT: return "invalid support (must be ascending, distinct, in range)";
+        case CS_ERR_NONFINITE: return "non-finite or non-positive scalar parameter";
+        case CS_ERR_CUDA: return "CUDA runtime error";
+        case CS_ERR_TIMEOUT: return "bounded device wait gave up";
+    }
+    return "unknown status";
+}
+
+}  // extern "C"

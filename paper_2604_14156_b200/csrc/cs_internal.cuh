@@ -1,0 +1,120 @@
+// Internal declarations shared by the library's translation units (not part of the C boundary).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "cs.h"
+
+namespace cs {
+
+constexpr int kMaxG = 128;        // groups per layer
+constexpr int kMaxM = 64;         // sketch rows
+constexpr int kMaxD = 8192;       // hidden size
+constexpr int kGatherThreads = 512;
+constexpr int kGatherMaxRows = 32;   // channel rows one gather CTA owns at most
+constexpr int kGatherMaxTokens = 16; // tokens per gather launch (scratch for partial sums)
+constexpr int kReduceGroups = 32;    // partial-sum groups of the deterministic cross-CTA reduction
+
+// Device status word values mirror cs_status (0 = ok).
+struct DeviceStatus {
+    int code;
+};
+
+}  // namespace cs
+
+struct cs_plan {
+    cs_config cfg;
+    int G;
+    int device;
+    int sm_count;
+    // device scratch
+    float *n_buf;      // [max_tokens, d]  normalised FFN input
+    float *y_buf;      // [max_tokens, m]
+    int32_t *sup_buf;  // [max_tokens, k]
+    float *z_buf;      // [max_tokens, k]
+    float *resid_buf;  // [max_tokens]
+    float *partial;    // [kGatherMaxTokens, nx_max, d] partial down-projections of the gather path
+    float *hbar;       // [d] mean prompt hidden state
+    float *colsum;     // [mean_row_blocks, d]
+    cs::DeviceStatus *status;  // device status word
+    float *x_host_in;  // [max_tokens, d] staging for the host-buffer entry point
+    float *x_host_out; // [max_tokens, d]
+    cudaEvent_t ev[2 * CS_STAGE_COUNT];  // start/stop per stage
+    int timing;
+    int stage_seen[CS_STAGE_COUNT];
+    int nx_max;
+    int mean_row_blocks;
+    int64_t launches;
+    char cuda_error[256];
+};
+
+namespace cs {
+
+cs_status record_cuda(cs_plan *plan, cudaError_t e, const char *what);
+
+#define CS_CUDA_TRY(plan, expr)                                                     \
+    do {                                                                            \
+        cudaError_t e_ = (expr);                                                    \
+        if (e_ != cudaSuccess) return ::cs::record_cuda((plan), e_, #expr);         \
+    } while (0)
+
+// Brackets one stage's launches with events when timing is enabled.
+struct StageTimer {
+    cs_plan *p; int stage; cudaStream_t st;
+    StageTimer(cs_plan *plan, int s, cudaStream_t stream) : p(plan), stage(s), st(stream) {
+        if (p->timing) cudaEventRecord(p->ev[2 * stage], st);
+    }
+    ~StageTimer() {
+        if (p->timing) { cudaEventRecord(p->ev[2 * stage + 1], st); p->stage_seen[stage] = 1; }
+    }
+};
+
+// Kernel launchers (each enqueues on `st`, bumps plan->launches, returns a status).
+cs_status launch_sketch(cs_plan *plan, const float *S, const float *x, const float *gamma, int B,
+                        float *y, float *n_out, cudaStream_t st);
+cs_status launch_recover(cs_plan *plan, const float *Phi, float mu, const float *y, int B,
+                         int32_t *support, float *z, float *resid, cudaStream_t st);
+cs_status launch_ffn_gather(cs_plan *plan, const cs_layer *layer, const float *h, const int32_t *support,
+                            int B, const float *residual, float *out, cudaStream_t st);
+cs_status launch_check_support(cs_plan *plan, const int32_t *support, int B, cudaStream_t st);
+cs_status launch_prompt_mean(cs_plan *plan, const void *H, int n, float *hbar, cudaStream_t st);
+
+// ---- small device helpers -------------------------------------------------------------------
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+// 16-byte read-only streaming load (weights are read once per step: keep them out of L1).
+__device__ __forceinline__ uint4 ldg_stream(const void *p) {
+    uint4 r;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w)
+                 : "l"(p));
+    return r;
+}
+
+__device__ __forceinline__ float bf16_lo(uint32_t u) { return __uint_as_float(u << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t u) { return __uint_as_float(u & 0xffff0000u); }
+
+// Widen one 16-byte chunk of weights to floats: 8 values for bf16, 4 for f32.
+template <typename WT> struct Chunk;
+template <> struct Chunk<__nv_bfloat16> {
+    static constexpr int kElems = 8;
+    __device__ static __forceinline__ void widen(const uint4 &q, float (&f)[8]) {
+        f[0] = bf16_lo(q.x); f[1] = bf16_hi(q.x); f[2] = bf16_lo(q.y); f[3] = bf16_hi(q.y);
+        f[4] = bf16_lo(q.z); f[5] = bf16_hi(q.z); f[6] = bf16_lo(q.w); f[7] = bf16_hi(q.w);
+    }
+};
+template <> struct Chunk<float> {
+    static constexpr int kElems = 4;
+    __device__ static __forceinline__ void widen(const uint4 &q, float (&f)[4]) {
+        f[0] = __uint_as_float(q.x); f[1] = __uint_as_float(q.y);
+        f[2] = __uint_as_float(q.z); f[3] = __uint_as_float(q.w);
+    }
+};
+
+}  // namespace cs

@@ -1,0 +1,247 @@
+// Actuator, small-batch regime: a gather GEMV that streams every active weight row exactly once.
+//
+// The k*b active channel rows of a token are split evenly over the CTAs of its grid row.  A CTA
+// owns a contiguous range of channel rows and does, for those rows only,
+//     a[c]      = silu(W_gate[c,:] . h) * (W_up[c,:] . h)
+//     partial[:] = sum_c a[c] * Wd_t[c,:]
+// so gate, up and down rows of a channel are consumed by the same CTA and nothing but the
+// d-vector of partial sums crosses CTAs.  Inside a CTA the hidden dimension is split over all
+// threads: thread i owns 16-byte chunk i (+512, ...) of every row, i.e. one coalesced 16-byte
+// load per row and matrix, with all rows of the CTA independent and in flight together.
+// The partial d-vectors are summed in a fixed order by reduce_partials_kernel (deterministic,
+// no atomics), which also adds the residual.
+#include "cs_internal.cuh"
+
+namespace cs {
+
+__device__ __forceinline__ float silu(float x) { return x / (1.f + __expf(-x)); }
+
+// CPT = 16-byte chunks per thread and row.
+template <typename WT, int CPT>
+__global__ void __launch_bounds__(kGatherThreads)
+ffn_gather_kernel(const WT *__restrict__ Wg, const WT *__restrict__ Wu, const WT *__restrict__ Wdt,
+                  const float *__restrict__ h, const int32_t *__restrict__ support, int d, int b, int k,
+                  float *__restrict__ partial) {
+    constexpr int E = Chunk<WT>::kElems;
+    constexpr int kWarps = kGatherThreads / 32;
+    __shared__ float red[2 * kGatherMaxRows][kWarps];
+    __shared__ float a_s[kGatherMaxRows];
+    __shared__ int chan_s[kGatherMaxRows];
+
+    const int t = blockIdx.y, nx = gridDim.x;
+    const int rows_total = k * b;
+    const int r_begin = (int)(((long long)rows_total * blockIdx.x) / nx);
+    const int r_end = (int)(((long long)rows_total * (blockIdx.x + 1)) / nx);
+    const int nrows = r_end - r_begin;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int chunks = d / E;
+
+    if (tid < nrows) {
+        const int c = r_begin + tid;
+        chan_s[tid] = support[(size_t)t * k + c / b] * b + c % b;
+    }
+    // this thread's slice of h
+    float hv[CPT][E];
+#pragma unroll
+    for (int j = 0; j < CPT; ++j) {
+        const int c = tid + j * kGatherThreads;
+#pragma unroll
+        for (int e = 0; e < E; e += 4) {
+            float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (c < chunks) v = *reinterpret_cast<const float4 *>(h + (size_t)t * d + (size_t)c * E + e);
+            hv[j][e] = v.x; hv[j][e + 1] = v.y; hv[j][e + 2] = v.z; hv[j][e + 3] = v.w;
+        }
+    }
+    __syncthreads();
+
+    // ---- gate / up: partial dot products of this thread's chunks, rows in batches of 8 loads
+    constexpr int RB = 4 / CPT > 0 ? 4 / CPT : 1;
+    for (int r0 = 0; r0 < nrows; r0 += RB) {
+        uint4 qg[RB][CPT], qu[RB][CPT];
+#pragma unroll
+        for (int r = 0; r < RB; ++r) {
+            const bool live = r0 + r < nrows;
+            const size_t base = live ? (size_t)chan_s[r0 + r] * d : 0;
+#pragma unroll
+            for (int j = 0; j < CPT; ++j) {
+                const int c = tid + j * kGatherThreads;
+                qg[r][j] = make_uint4(0, 0, 0, 0); qu[r][j] = make_uint4(0, 0, 0, 0);
+                if (live && c < chunks) {
+                    qg[r][j] = ldg_stream(Wg + base + (size_t)c * E);
+                    qu[r][j] = ldg_stream(Wu + base + (size_t)c * E);
+                }
+            }
+        }
+#pragma unroll
+        for (int r = 0; r < RB; ++r) {
+            float g = 0.f, u = 0.f;
+#pragma unroll
+            for (int j = 0; j < CPT; ++j) {
+                float wg[E], wu[E];
+                Chunk<WT>::widen(qg[r][j], wg);
+                Chunk<WT>::widen(qu[r][j], wu);
+#pragma unroll
+                for (int e = 0; e < E; ++e) { g = fmaf(wg[e], hv[j][e], g); u = fmaf(wu[e], hv[j][e], u); }
+            }
+            g = warp_sum(g); u = warp_sum(u);
+            if (lane == 0 && r0 + r < nrows) { red[2 * (r0 + r)][warp] = g; red[2 * (r0 + r) + 1][warp] = u; }
+        }
+    }
+    __syncthreads();
+    if (tid < nrows) {
+        float g = 0.f, u = 0.f;
+#pragma unroll
+        for (int w = 0; w < kWarps; ++w) { g += red[2 * tid][w]; u += red[2 * tid + 1][w]; }
+        a_s[tid] = silu(g) * u;
+    }
+    __syncthreads();
+
+    // ---- down: this CTA's contribution to every output column, rows in batches of 8
+    float acc[CPT][E];
+#pragma unroll
+    for (int j = 0; j < CPT; ++j)
+#pragma unroll
+        for (int e = 0; e < E; ++e) acc[j][e] = 0.f;
+    constexpr int DB = 8 / CPT > 0 ? 8 / CPT : 1;
+    for (int r0 = 0; r0 < nrows; r0 += DB) {
+        uint4 q[DB][CPT];
+#pragma unroll
+        for (int r = 0; r < DB; ++r) {
+            const bool live = r0 + r < nrows;
+            const size_t base = live ? (size_t)chan_s[r0 + r] * d : 0;
+#pragma unroll
+            for (int j = 0; j < CPT; ++j) {
+                const int c = tid + j * kGatherThreads;
+                q[r][j] = make_uint4(0, 0, 0, 0);
+                if (live && c < chunks) q[r][j] = ldg_stream(Wdt + base + (size_t)c * E);
+            }
+        }
+#pragma unroll
+        for (int r = 0; r < DB; ++r) {
+            const float a = r0 + r < nrows ? a_s[r0 + r] : 0.f;
+#pragma unroll
+            for (int j = 0; j < CPT; ++j) {
+                float w[E];
+                Chunk<WT>::widen(q[r][j], w);
+#pragma unroll
+                for (int e = 0; e < E; ++e) acc[j][e] = fmaf(a, w[e], acc[j][e]);
+            }
+        }
+    }
+    float *dst = partial + ((size_t)t * nx + blockIdx.x) * d;
+#pragma unroll
+    for (int j = 0; j < CPT; ++j) {
+        const int c = tid + j * kGatherThreads;
+        if (c < chunks) {
+#pragma unroll
+            for (int e = 0; e < E; e += 4)
+                *reinterpret_cast<float4 *>(dst + (size_t)c * E + e) =
+                    make_float4(acc[j][e], acc[j][e + 1], acc[j][e + 2], acc[j][e + 3]);
+        }
+    }
+}
+
+// out[t, :] = residual[t, :] + sum_{p < nx} partial[t, p, :], p ascending within fixed groups.
+// CTA = 32 float4 columns x kReduceGroups partial groups; a thread sums the partials p with
+// p % kReduceGroups == its group, then the groups are folded in index order through shared memory.
+__global__ void __launch_bounds__(32 * kReduceGroups)
+reduce_partials_kernel(const float *__restrict__ partial, int nx, int d, const float *__restrict__ residual,
+                       float *__restrict__ out) {
+    __shared__ float4 fold[kReduceGroups][32];
+    const int t = blockIdx.y;
+    const int col = blockIdx.x * 32 + (threadIdx.x & 31);  // float4 column
+    const int grp = threadIdx.x >> 5;
+    const int cols = d >> 2;
+    float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (col < cols) {
+        const float4 *src = reinterpret_cast<const float4 *>(partial + (size_t)t * nx * d) + col;
+        for (int p = grp; p < nx; p += kReduceGroups) {
+            const float4 v = src[(size_t)p * cols];
+            s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
+        }
+    }
+    fold[grp][threadIdx.x & 31] = s;
+    __syncthreads();
+    if (grp == 0 && col < cols) {
+        float4 r = residual != nullptr ? reinterpret_cast<const float4 *>(residual + (size_t)t * d)[col]
+                                       : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int g = 0; g < kReduceGroups; ++g) {
+            const float4 v = fold[g][threadIdx.x & 31];
+            r.x += v.x; r.y += v.y; r.z += v.z; r.w += v.w;
+        }
+        reinterpret_cast<float4 *>(out + (size_t)t * d)[col] = r;
+    }
+}
+
+// Device-side validation of supports (ascending, distinct, in range); records CS_ERR_SUPPORT.
+__global__ void check_support_kernel(const int32_t *__restrict__ support, int B, int k, int G,
+                                     DeviceStatus *status) {
+    const int t = blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= B) return;
+    int prev = -1;
+    bool ok = true;
+    for (int c = 0; c < k; ++c) {
+        const int g = support[(size_t)t * k + c];
+        ok = ok && g > prev && g < G;
+        prev = g;
+    }
+    if (!ok) atomicCAS(&status->code, 0, (int)CS_ERR_SUPPORT);
+}
+
+cs_status launch_check_support(cs_plan *plan, const int32_t *support, int B, cudaStream_t st) {
+    check_support_kernel<<<(B + 127) / 128, 128, 0, st>>>(support, B, plan->cfg.k, plan->G, plan->status);
+    plan->launches++;
+    CS_CUDA_TRY(plan, cudaGetLastError());
+    return CS_OK;
+}
+
+template <typename WT>
+static cs_status gather_typed(cs_plan *plan, const cs_layer *L, const float *h, const int32_t *support,
+                              int B, const float *residual, float *out, cudaStream_t st) {
+    const cs_config &c = plan->cfg;
+    constexpr int E = Chunk<WT>::kElems;
+    const int rows_total = c.k * c.group;
+    const int cpt = (c.d / E + kGatherThreads - 1) / kGatherThreads;
+    const WT *Wg = static_cast<const WT *>(L->W_gate), *Wu = static_cast<const WT *>(L->W_up),
+             *Wd = static_cast<const WT *>(L->Wd_t);
+    for (int t0 = 0; t0 < B; t0 += kGatherMaxTokens) {
+        const int nb = min(kGatherMaxTokens, B - t0);
+        // one CTA per SM when a single token is in flight, never more than kGatherMaxRows rows per CTA
+        int nx = max(plan->sm_count / nb, (rows_total + kGatherMaxRows - 1) / kGatherMaxRows);
+        nx = max(1, min(nx, min(rows_total, plan->nx_max)));
+        dim3 grid(nx, nb);
+        const float *hp = h + (size_t)t0 * c.d;
+        const int32_t *sp = support + (size_t)t0 * c.k;
+#define CS_GATHER_CASE(N)                                                                          \
+    ffn_gather_kernel<WT, N><<<grid, kGatherThreads, 0, st>>>(Wg, Wu, Wd, hp, sp, c.d, c.group, c.k, \
+                                                              plan->partial)
+        {
+            StageTimer timer(plan, CS_STAGE_EXEC, st);
+            if (cpt <= 1) CS_GATHER_CASE(1);
+            else if (cpt <= 2) CS_GATHER_CASE(2);
+            else CS_GATHER_CASE(4);
+        }
+#undef CS_GATHER_CASE
+        plan->launches++;
+        CS_CUDA_TRY(plan, cudaGetLastError());
+        dim3 rgrid((c.d / 4 + 31) / 32, nb);
+        {
+            StageTimer timer(plan, CS_STAGE_REDUCE, st);
+            reduce_partials_kernel<<<rgrid, 32 * kReduceGroups, 0, st>>>(
+                plan->partial, nx, c.d, residual ? residual + (size_t)t0 * c.d : nullptr, out + (size_t)t0 * c.d);
+        }
+        plan->launches++;
+        CS_CUDA_TRY(plan, cudaGetLastError());
+    }
+    return CS_OK;
+}
+
+cs_status launch_ffn_gather(cs_plan *plan, const cs_layer *layer, const float *h, const int32_t *support,
+                            int B, const float *residual, float *out, cudaStream_t st) {
+    if (plan->cfg.w_dtype == CS_BF16)
+        return gather_typed<__nv_bfloat16>(plan, layer, h, support, B, residual, out, st);
+    return gather_typed<float>(plan, layer, h, support, B, residual, out, st);
+}
+
+}  // namespace cs

@@ -1,0 +1,249 @@
+"""GPU parity: the CUDA library (through the C boundary) against the fp64 CPU oracle on the same
+seeded inputs.  Tolerances are those of tests/parity_util.py."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2604_14156_b200 as cs
+from gen import rng, workloads as W
+from parity_util import (GAP_TOL, OUT_TOL, Z_TOL, compare_layer_step, device_layer, make_plan, rel)
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def _layer(cfg, layer=0, **kw):
+    return W.make_layer(cfg, layer, device=DEV, **kw)
+
+
+# ------------------------------------------------------------------ single entry points
+@pytest.mark.parametrize("name,B", [("tiny_f32", 4), ("l2_7b_b1", 1), ("l2_7b_b64", 64), ("l3_8b_stack", 5)])
+def test_sketch_matches_oracle(name, B):
+    cfg = W.CONFIGS[name]
+    A = W.make_probe(cfg)
+    Phi = rng.normal(cfg.seed, (W.T_PHI, 0), (cfg.m, cfg.G), dtype=torch.float32, scale=cfg.m ** -0.5)
+    S = (Phi.double() @ A).float()
+    h = W.make_tokens(cfg, A, B=B).h
+    plan = make_plan(cfg, max_tokens=max(B, 1))
+    y = cs.cs_sketch(plan, S.to(DEV), h.to(DEV)).cpu().numpy()
+    ref = oracle.sketch(S, h)
+    assert rel(y, ref) <= 1e-5
+    assert np.abs(y - ref).max() <= 1e-5 * np.abs(ref).max()
+
+
+@pytest.mark.parametrize("name", ["tiny_f32", "l2_7b_b64", "l3_8b_stack", "l2_13b_prompt"])
+def test_recover_matches_oracle(name):
+    cfg = W.CONFIGS[name]
+    B = 48
+    Phi = rng.normal(cfg.seed, (W.T_PHI, 0), (cfg.m, cfg.G), dtype=torch.float32, scale=cfg.m ** -0.5)
+    mu = W.spectral_step(Phi)
+    y = rng.normal(cfg.seed, (77,), (B, cfg.m), dtype=torch.float32)
+    plan = make_plan(cfg, max_tokens=B)
+    sup, z, resid = cs.cs_recover(plan, Phi.to(DEV), mu, y.to(DEV))
+    sup = sup.cpu().numpy(); z = z.cpu().numpy(); resid = resid.cpu().numpy()
+    excused = 0
+    for t in range(B):
+        ref = oracle.iht(Phi, y[t], cfg.k, cfg.T, mu)
+        if np.array_equal(sup[t], ref.support):
+            assert rel(z[t], ref.z[ref.support]) <= Z_TOL
+            assert abs(resid[t] - ref.resid) <= 1e-4 * max(1.0, ref.resid)
+        else:
+            assert ref.min_gap <= GAP_TOL
+            excused += 1
+    assert excused <= 2
+
+
+def test_recover_edge_cases():
+    """T = 0, k = G, k = 1, all-zero sketch (every comparison a tie), exact ties between groups."""
+    cfg = W.CONFIGS["tiny_f32"]
+    Phi = rng.normal(5, (1,), (cfg.m, cfg.G), dtype=torch.float32, scale=cfg.m ** -0.5)
+    mu = W.spectral_step(Phi)
+    y = rng.normal(5, (2,), (3, cfg.m), dtype=torch.float32)
+    for k, T in [(4, 0), (16, 10), (1, 10), (15, 3)]:
+        c = cfg.with_(k=k, T=T)
+        plan = make_plan(c, max_tokens=3)
+        sup, z, resid = cs.cs_recover(plan, Phi.to(DEV), mu, y.to(DEV))
+        for t in range(3):
+            ref = oracle.iht(Phi, y[t], k, T, mu)
+            assert np.array_equal(sup[t].cpu().numpy(), ref.support), (k, T)
+            assert rel(z[t].cpu().numpy(), ref.z[ref.support]) <= Z_TOL or not ref.z.any()
+            assert abs(resid[t].item() - ref.resid) <= 1e-4 * max(1.0, ref.resid)
+    # y = 0: v is identically zero, the order falls back to the index -> 0..k-1
+    plan = make_plan(cfg, max_tokens=2)
+    sup, z, resid = cs.cs_recover(plan, Phi.to(DEV), mu, torch.zeros(2, cfg.m, device=DEV))
+    assert sup.cpu().tolist() == [[0, 1, 2, 3]] * 2 and not z.any() and not resid.any()
+    # duplicated columns give exact ties: the lower index must win on both sides
+    Phi2 = Phi.clone(); Phi2[:, 9] = Phi2[:, 2]; Phi2[:, 12] = -Phi2[:, 5]
+    sup, z, _ = cs.cs_recover(plan, Phi2.to(DEV), W.spectral_step(Phi2), y[:2].to(DEV))
+    for t in range(2):
+        ref = oracle.iht(Phi2, y[t], cfg.k, cfg.T, W.spectral_step(Phi2))
+        if ref.min_gap > GAP_TOL or not ref.z.any():
+            assert np.array_equal(sup[t].cpu().numpy(), ref.support)
+
+
+@pytest.mark.parametrize("name,B", [("tiny_f32", 4), ("l2_7b_b1", 1), ("l2_7b_b64", 3)])
+def test_ffn_exec_matches_oracle_on_given_supports(name, B):
+    cfg = W.CONFIGS[name]
+    L = _layer(cfg)
+    Lc = L.to("cpu")
+    tk = W.make_tokens(cfg, L.A, B=B)
+    plan = make_plan(cfg, max_tokens=B)
+    lay = device_layer(plan, L)
+    res = rng.normal(cfg.seed, (78,), (B, cfg.d), dtype=torch.float32)
+    out = cs.cs_ffn_exec(plan, lay, tk.h.to(DEV), tk.planted.to(DEV), residual=res.to(DEV)).cpu().numpy()
+    out0 = cs.cs_ffn_exec(plan, lay, tk.h.to(DEV), tk.planted.to(DEV)).cpu().numpy()
+    assert plan.device_status() == 0
+    for t in range(B):
+        ref = oracle.ffn(Lc.W_gate, Lc.W_up, Lc.Wd_t, cfg.group, tk.h[t], tk.planted[t])
+        assert rel(out0[t], ref) <= OUT_TOL[cfg.w_dtype]
+        assert rel(out[t], ref + res[t].double().numpy()) <= OUT_TOL[cfg.w_dtype]
+
+
+def test_ffn_exec_all_groups_is_the_dense_ffn():
+    cfg = W.CONFIGS["tiny_f32"].with_(k=16)
+    L = _layer(cfg)
+    tk = W.make_tokens(cfg, L.A, B=2)
+    plan = make_plan(cfg, max_tokens=2)
+    sup = torch.arange(16, dtype=torch.int32).repeat(2, 1)
+    out = cs.cs_ffn_exec(plan, device_layer(plan, L), tk.h.to(DEV), sup.to(DEV)).cpu().double().numpy()
+    Wg, Wu, Wdt = (w.cpu().double().numpy() for w in (L.W_gate, L.W_up, L.Wd_t))
+    for t in range(2):
+        h = tk.h[t].double().numpy()
+        g = Wg @ h; u = Wu @ h
+        dense = ((g / (1 + np.exp(-g))) * u) @ Wdt
+        assert rel(out[t], dense) <= 1e-5
+
+
+def test_ffn_exec_flags_invalid_supports():
+    cfg = W.CONFIGS["tiny_f32"]
+    L = _layer(cfg)
+    plan = make_plan(cfg, max_tokens=2)
+    lay = device_layer(plan, L)
+    h = torch.zeros(2, cfg.d, device=DEV)
+    good = torch.tensor([[0, 1, 2, 3], [4, 5, 6, 15]], dtype=torch.int32, device=DEV)
+    cs.cs_ffn_exec(plan, lay, h, good)
+    assert plan.device_status() == 0
+    # unsorted but in range: flagged, and harmless to execute
+    bad = torch.tensor([[0, 1, 2, 3], [4, 6, 5, 15]], dtype=torch.int32, device=DEV)
+    cs.cs_ffn_exec(plan, lay, h, bad)
+    assert plan.device_status() == 4
+    assert plan.device_status() == 0  # reading clears it
+
+
+def test_call_errors_come_back_as_codes():
+    cfg = W.CONFIGS["tiny_f32"]
+    plan = make_plan(cfg, max_tokens=2)
+    S = torch.zeros(cfg.m, cfg.d, device=DEV)
+    with pytest.raises(cs.CSError) as e:
+        cs.cs_sketch(plan, S, torch.zeros(3, cfg.d, device=DEV))  # B > max_tokens
+    assert e.value.code == 2
+    with pytest.raises(cs.CSError) as e:
+        cs.cs_recover(plan, torch.zeros(cfg.m, cfg.G, device=DEV), float("nan"), torch.zeros(1, cfg.m, device=DEV))
+    assert e.value.code == 5
+    misaligned = torch.zeros(2 * cfg.d + 1, device=DEV)[1:1 + cfg.d].view(1, cfg.d)  # 4-byte offset
+    with pytest.raises(cs.CSError) as e:
+        cs.cs_sketch(plan, S, misaligned)
+    assert e.value.code == 3
+
+
+# ------------------------------------------------------------------ whole step, the five workloads
+@pytest.mark.parametrize("seed_offset", [0, 1000, 2000])
+@pytest.mark.parametrize("name", ["tiny_f32", "l2_7b_b1", "l2_7b_b64"])
+def test_layer_step_parity(name, seed_offset):
+    cfg = W.CONFIGS[name]
+    cfg = cfg.with_(index=cfg.index + seed_offset)
+    L = _layer(cfg)
+    tk = W.make_tokens(cfg, L.A)
+    plan = make_plan(cfg)
+    rep, _, _ = compare_layer_step(cfg, L, plan, tk.h)
+    assert rep.excused <= max(1, cfg.B // 16)
+    print(f"{name}+{seed_offset}: {rep}")
+
+
+def test_layer_step_literal_unit_step_tiny():
+    """The tiny workload with the literal mu = 1 (diverging iterates): parity must still hold."""
+    cfg = W.CONFIGS["tiny_f32"]
+    L = _layer(cfg, literal_mu=1.0)
+    tk = W.make_tokens(cfg, L.A)
+    rep, _, _ = compare_layer_step(cfg, L, make_plan(cfg), tk.h)
+    print(rep)
+
+
+@pytest.mark.parametrize("shape", [
+    dict(d=192, d_ff=64 * 5, group=64, m=5, k=2, B=3),         # nothing a multiple of 32
+    dict(d=8192, d_ff=128 * 7, group=128, m=64, k=7, B=2),     # widest rows, k = G
+    dict(d=1024, d_ff=128 * 128, group=128, m=33, k=1, B=17),  # most groups, ragged token tail
+    dict(d=320, d_ff=64 * 33, group=64, m=17, k=9, B=37),
+])
+@pytest.mark.parametrize("w", ["f32", "bf16"])
+def test_layer_step_ragged_shapes(shape, w):
+    cfg = W.CONFIGS["l3_8b_stack"].with_(n_layers=1, w_dtype=w, T=6, **shape)
+    L = _layer(cfg)
+    tk = W.make_tokens(cfg, L.A)
+    rep, _, _ = compare_layer_step(cfg, L, make_plan(cfg), tk.h)
+    print(shape, w, rep)
+
+
+def test_layer_step_in_place_and_without_aux_outputs():
+    cfg = W.CONFIGS["l3_8b_stack"].with_(n_layers=1, d=512, d_ff=2048, m=16, k=4, B=6)
+    L = _layer(cfg)
+    tk = W.make_tokens(cfg, L.A)
+    plan = make_plan(cfg)
+    lay = device_layer(plan, L)
+    x = tk.h.to(DEV)
+    ref_out, *_ = cs.cs_layer_step(plan, lay, x)
+    y = x.clone()
+    cs.cs_layer_step(plan, lay, y, x_out=y, want_aux=False)
+    assert torch.equal(y, ref_out)
+    again, *_ = cs.cs_layer_step(plan, lay, x)
+    assert torch.equal(again, ref_out)  # deterministic: no atomics on the path
+
+
+def test_stack_parity_teacher_forced_and_chained():
+    """32 Llama-3-8B-shaped layers, batch 32: (i) every layer fed the oracle's input for that
+    layer; (ii) the library's own chained output against the oracle's chain, replayed with the
+    library's supports where a near-tie was excused."""
+    cfg = W.CONFIGS["l3_8b_stack"]
+    plan = make_plan(cfg)
+    L0 = _layer(cfg, 0)
+    x_ref = W.make_tokens(cfg, L0.A).h.double().numpy()
+    x_gpu = torch.from_numpy(x_ref).float().to(DEV)
+    excused = 0
+    worst = 0.0
+    for layer in range(cfg.n_layers):
+        L = L0 if layer == 0 else _layer(cfg, layer)
+        x_in = torch.from_numpy(x_ref).float()      # teacher forcing: oracle's stream, as stored f32
+        rep, ref_out, _ = compare_layer_step(cfg, L, plan, x_in)
+        excused += rep.excused
+        worst = max(worst, rep.max_out_err)
+        # chained: the library's own residual stream
+        lay = device_layer(plan, L)
+        cs.cs_layer_step(plan, lay, x_gpu, x_out=x_gpu, want_aux=False)
+        x_ref = ref_out
+        del L, lay
+    torch.cuda.synchronize()
+    chain_err = rel(x_gpu.cpu().numpy(), x_ref)
+    print(f"stack: excused {excused}/{cfg.B * cfg.n_layers}, worst layer err {worst:.2e}, chained err {chain_err:.2e}")
+    assert excused <= 8
+    if excused == 0:
+        assert chain_err <= OUT_TOL["bf16"]
+
+
+@pytest.mark.parametrize("k", W.PROMPT_K_SWEEP)
+def test_prompt_support_parity(k):
+    cfg = W.CONFIGS["l2_13b_prompt"].with_(k=k)
+    A = W.make_probe(cfg)
+    Phi = rng.normal(cfg.seed, (W.T_PHI, 0), (cfg.m, cfg.G), dtype=torch.float32, scale=cfg.m ** -0.5)
+    S = (Phi.double() @ A).float()
+    mu = W.spectral_step(Phi)
+    H = W.make_tokens(cfg, A).h
+    plan = make_plan(cfg)
+    sup, z, resid = cs.cs_prompt_support(plan, S.to(DEV), Phi.to(DEV), mu, H.to(DEV))
+    ybar, ref = oracle.prompt_support(S, Phi, H, k, cfg.T, mu)
+    sup = sup.cpu().numpy()
+    if ref.min_gap > GAP_TOL:
+        assert np.array_equal(sup, ref.support)
+    if np.array_equal(sup, ref.support):
+        assert rel(z.cpu().numpy(), ref.z[ref.support]) <= Z_TOL
+        assert abs(resid.item() - ref.resid) <= 1e-4 * max(1.0, ref.resid)
