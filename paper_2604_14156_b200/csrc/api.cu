@@ -67,6 +67,7 @@ cs_status cs_plan_create(const cs_config *cfg, cs_plan **out) {
     for (int i = 0; i < 2 * CS_STAGE_COUNT; ++i)
         if (e == cudaSuccess) e = cudaEventCreate(&p->ev[i]);
     if (e == cudaSuccess) e = cudaMemset(p->status, 0, sizeof(DeviceStatus));
+    if (e == cudaSuccess && prepare_ffn_gather(p) != CS_OK) e = cudaErrorUnknown;
     if (e != cudaSuccess) {
         cs_plan_destroy(p);
         return CS_ERR_CUDA;

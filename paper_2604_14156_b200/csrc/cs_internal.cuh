@@ -78,6 +78,7 @@ cs_status launch_recover(cs_plan *plan, const float *Phi, float mu, const float 
                          int32_t *support, float *z, float *resid, cudaStream_t st);
 cs_status launch_ffn_gather(cs_plan *plan, const cs_layer *layer, const float *h, const int32_t *support,
                             int B, const float *residual, float *out, cudaStream_t st);
+cs_status prepare_ffn_gather(cs_plan *plan);
 cs_status launch_check_support(cs_plan *plan, const int32_t *support, int B, cudaStream_t st);
 cs_status launch_prompt_mean(cs_plan *plan, const void *H, int n, float *hbar, cudaStream_t st);
 

@@ -6,8 +6,14 @@
 //     partial[:] = sum_c a[c] * Wd_t[c,:]
 // so gate, up and down rows of a channel are consumed by the same CTA and nothing but the
 // d-vector of partial sums crosses CTAs.  Inside a CTA the hidden dimension is split over all
-// threads: thread i owns 16-byte chunk i (+512, ...) of every row, i.e. one coalesced 16-byte
-// load per row and matrix, with all rows of the CTA independent and in flight together.
+// threads: thread i owns 16-byte chunk i (+512, ...) of every row.
+//
+// The kernel is a pure HBM stream (3 * rows * d weight elements, each used once), so what matters
+// is bytes in flight.  Every thread runs its own cp.async ring: it copies its 16-byte chunks of
+// the next rows into its private slots of a shared-memory ring (L2 -> shared, bypassing L1 and
+// registers), up to kRingBytes per CTA ahead of use, and reads back only what it copied itself,
+// so the ring needs no barrier at all.  The down rows are already in flight while the gate/up
+// results are being folded across warps.
 // The partial d-vectors are summed in a fixed order by reduce_partials_kernel (deterministic,
 // no atomics), which also adds the residual.
 #include "cs_internal.cuh"
@@ -16,7 +22,20 @@ namespace cs {
 
 __device__ __forceinline__ float silu(float x) { return x / (1.f + __expf(-x)); }
 
-// CPT = 16-byte chunks per thread and row.
+constexpr int kRingBytes = 192 * 1024;
+constexpr int kItemBytes = 2 * 16 * kGatherThreads;  // two rows' worth of one chunk per thread
+
+__device__ __forceinline__ void cp_async16(void *smem_dst, const void *gmem_src) {
+    const uint32_t s = static_cast<uint32_t>(__cvta_generic_to_shared(smem_dst));
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(s), "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() {
+    asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+
+// CPT = 16-byte chunks per thread and row.  Ring item i: i < nrows -> (gate row i, up row i);
+// i >= nrows -> (down row 2(i-nrows), down row 2(i-nrows)+1).
 template <typename WT, int CPT>
 __global__ void __launch_bounds__(kGatherThreads)
 ffn_gather_kernel(const WT *__restrict__ Wg, const WT *__restrict__ Wu, const WT *__restrict__ Wdt,
@@ -24,8 +43,10 @@ ffn_gather_kernel(const WT *__restrict__ Wg, const WT *__restrict__ Wu, const WT
                   float *__restrict__ partial) {
     constexpr int E = Chunk<WT>::kElems;
     constexpr int kWarps = kGatherThreads / 32;
+    constexpr int NS = kRingBytes / (kItemBytes * CPT);  // ring stages
+    extern __shared__ __align__(16) uint4 ring[];        // [NS][2][CPT][kGatherThreads]
     __shared__ float red[2 * kGatherMaxRows][kWarps];
-    __shared__ float a_s[kGatherMaxRows];
+    __shared__ float a_s[kGatherMaxRows + 1];
     __shared__ int chan_s[kGatherMaxRows];
 
     const int t = blockIdx.y, nx = gridDim.x;
@@ -33,6 +54,7 @@ ffn_gather_kernel(const WT *__restrict__ Wg, const WT *__restrict__ Wu, const WT
     const int r_begin = (int)(((long long)rows_total * blockIdx.x) / nx);
     const int r_end = (int)(((long long)rows_total * (blockIdx.x + 1)) / nx);
     const int nrows = r_end - r_begin;
+    const int nitems = nrows + (nrows + 1) / 2;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int chunks = d / E;
 
@@ -40,6 +62,40 @@ ffn_gather_kernel(const WT *__restrict__ Wg, const WT *__restrict__ Wu, const WT
         const int c = r_begin + tid;
         chan_s[tid] = support[(size_t)t * k + c / b] * b + c % b;
     }
+    if (tid == 0) a_s[nrows] = 0.f;  // pad for an odd last down pair
+    __syncthreads();
+
+    auto slot = [&](int stage, int half, int j) -> uint4 * {
+        return ring + (((size_t)stage * 2 + half) * CPT + j) * kGatherThreads + tid;
+    };
+    auto issue = [&](int i) {
+        if (i < nitems) {
+            const WT *p0, *p1;
+            bool two = true;
+            if (i < nrows) {
+                const size_t base = (size_t)chan_s[i] * d;
+                p0 = Wg + base; p1 = Wu + base;
+            } else {
+                const int r = 2 * (i - nrows);
+                two = r + 1 < nrows;
+                p0 = Wdt + (size_t)chan_s[r] * d;
+                p1 = Wdt + (size_t)chan_s[two ? r + 1 : r] * d;
+            }
+            const int stage = i % NS;
+#pragma unroll
+            for (int j = 0; j < CPT; ++j) {
+                const int c = tid + j * kGatherThreads;
+                if (c < chunks) {
+                    cp_async16(slot(stage, 0, j), p0 + (size_t)c * E);
+                    if (two) cp_async16(slot(stage, 1, j), p1 + (size_t)c * E);
+                }
+            }
+        }
+        cp_async_commit();  // one group per item, empty past the end, so the wait count stays fixed
+    };
+#pragma unroll 1
+    for (int i = 0; i < NS; ++i) issue(i);
+
     // this thread's slice of h
     float hv[CPT][E];
 #pragma unroll
@@ -52,40 +108,27 @@ ffn_gather_kernel(const WT *__restrict__ Wg, const WT *__restrict__ Wu, const WT
             hv[j][e] = v.x; hv[j][e + 1] = v.y; hv[j][e + 2] = v.z; hv[j][e + 3] = v.w;
         }
     }
-    __syncthreads();
 
-    // ---- gate / up: partial dot products of this thread's chunks, rows in batches of 8 loads
-    constexpr int RB = 4 / CPT > 0 ? 4 / CPT : 1;
-    for (int r0 = 0; r0 < nrows; r0 += RB) {
-        uint4 qg[RB][CPT], qu[RB][CPT];
+    // ---- gate / up rows
+#pragma unroll 1
+    for (int i = 0; i < nrows; ++i) {
+        cp_async_wait<NS - 1>();
+        const int stage = i % NS;
+        float g = 0.f, u = 0.f;
 #pragma unroll
-        for (int r = 0; r < RB; ++r) {
-            const bool live = r0 + r < nrows;
-            const size_t base = live ? (size_t)chan_s[r0 + r] * d : 0;
-#pragma unroll
-            for (int j = 0; j < CPT; ++j) {
-                const int c = tid + j * kGatherThreads;
-                qg[r][j] = make_uint4(0, 0, 0, 0); qu[r][j] = make_uint4(0, 0, 0, 0);
-                if (live && c < chunks) {
-                    qg[r][j] = ldg_stream(Wg + base + (size_t)c * E);
-                    qu[r][j] = ldg_stream(Wu + base + (size_t)c * E);
-                }
-            }
-        }
-#pragma unroll
-        for (int r = 0; r < RB; ++r) {
-            float g = 0.f, u = 0.f;
-#pragma unroll
-            for (int j = 0; j < CPT; ++j) {
+        for (int j = 0; j < CPT; ++j) {
+            const int c = tid + j * kGatherThreads;
+            if (c < chunks) {
                 float wg[E], wu[E];
-                Chunk<WT>::widen(qg[r][j], wg);
-                Chunk<WT>::widen(qu[r][j], wu);
+                Chunk<WT>::widen(*slot(stage, 0, j), wg);
+                Chunk<WT>::widen(*slot(stage, 1, j), wu);
 #pragma unroll
                 for (int e = 0; e < E; ++e) { g = fmaf(wg[e], hv[j][e], g); u = fmaf(wu[e], hv[j][e], u); }
             }
-            g = warp_sum(g); u = warp_sum(u);
-            if (lane == 0 && r0 + r < nrows) { red[2 * (r0 + r)][warp] = g; red[2 * (r0 + r) + 1][warp] = u; }
         }
+        issue(i + NS);  // refill the slot just consumed (after its values were used above)
+        g = warp_sum(g); u = warp_sum(u);
+        if (lane == 0) { red[2 * i][warp] = g; red[2 * i + 1][warp] = u; }
     }
     __syncthreads();
     if (tid < nrows) {
@@ -96,38 +139,37 @@ ffn_gather_kernel(const WT *__restrict__ Wg, const WT *__restrict__ Wu, const WT
     }
     __syncthreads();
 
-    // ---- down: this CTA's contribution to every output column, rows in batches of 8
+    // ---- down rows, two per ring item
     float acc[CPT][E];
 #pragma unroll
     for (int j = 0; j < CPT; ++j)
 #pragma unroll
         for (int e = 0; e < E; ++e) acc[j][e] = 0.f;
-    constexpr int DB = 8 / CPT > 0 ? 8 / CPT : 1;
-    for (int r0 = 0; r0 < nrows; r0 += DB) {
-        uint4 q[DB][CPT];
+#pragma unroll 1
+    for (int i = nrows; i < nitems; ++i) {
+        cp_async_wait<NS - 1>();
+        const int stage = i % NS;
+        const int r = 2 * (i - nrows);
+        const float a0 = a_s[r], a1 = a_s[r + 1];
+        const bool two = r + 1 < nrows;
 #pragma unroll
-        for (int r = 0; r < DB; ++r) {
-            const bool live = r0 + r < nrows;
-            const size_t base = live ? (size_t)chan_s[r0 + r] * d : 0;
+        for (int j = 0; j < CPT; ++j) {
+            const int c = tid + j * kGatherThreads;
+            if (c < chunks) {
+                float w0[E], w1[E];
+                Chunk<WT>::widen(*slot(stage, 0, j), w0);
 #pragma unroll
-            for (int j = 0; j < CPT; ++j) {
-                const int c = tid + j * kGatherThreads;
-                q[r][j] = make_uint4(0, 0, 0, 0);
-                if (live && c < chunks) q[r][j] = ldg_stream(Wdt + base + (size_t)c * E);
+                for (int e = 0; e < E; ++e) acc[j][e] = fmaf(a0, w0[e], acc[j][e]);
+                if (two) {
+                    Chunk<WT>::widen(*slot(stage, 1, j), w1);
+#pragma unroll
+                    for (int e = 0; e < E; ++e) acc[j][e] = fmaf(a1, w1[e], acc[j][e]);
+                }
             }
         }
-#pragma unroll
-        for (int r = 0; r < DB; ++r) {
-            const float a = r0 + r < nrows ? a_s[r0 + r] : 0.f;
-#pragma unroll
-            for (int j = 0; j < CPT; ++j) {
-                float w[E];
-                Chunk<WT>::widen(q[r][j], w);
-#pragma unroll
-                for (int e = 0; e < E; ++e) acc[j][e] = fmaf(a, w[e], acc[j][e]);
-            }
-        }
+        issue(i + NS);
     }
+    cp_async_wait<0>();
     float *dst = partial + ((size_t)t * nx + blockIdx.x) * d;
 #pragma unroll
     for (int j = 0; j < CPT; ++j) {
@@ -155,7 +197,18 @@ reduce_partials_kernel(const float *__restrict__ partial, int nx, int d, const f
     float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
     if (col < cols) {
         const float4 *src = reinterpret_cast<const float4 *>(partial + (size_t)t * nx * d) + col;
-        for (int p = grp; p < nx; p += kReduceGroups) {
+        // partials p = grp, grp + 32, ...: loads issued four at a time, added in index order
+        int p = grp;
+        for (; p + 3 * kReduceGroups < nx; p += 4 * kReduceGroups) {
+            const float4 v0 = src[(size_t)p * cols], v1 = src[(size_t)(p + kReduceGroups) * cols],
+                         v2 = src[(size_t)(p + 2 * kReduceGroups) * cols],
+                         v3 = src[(size_t)(p + 3 * kReduceGroups) * cols];
+            s.x += v0.x; s.y += v0.y; s.z += v0.z; s.w += v0.w;
+            s.x += v1.x; s.y += v1.y; s.z += v1.z; s.w += v1.w;
+            s.x += v2.x; s.y += v2.y; s.z += v2.z; s.w += v2.w;
+            s.x += v3.x; s.y += v3.y; s.z += v3.z; s.w += v3.w;
+        }
+        for (; p < nx; p += kReduceGroups) {
             const float4 v = src[(size_t)p * cols];
             s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
         }
@@ -213,9 +266,9 @@ static cs_status gather_typed(cs_plan *plan, const cs_layer *L, const float *h, 
         dim3 grid(nx, nb);
         const float *hp = h + (size_t)t0 * c.d;
         const int32_t *sp = support + (size_t)t0 * c.k;
-#define CS_GATHER_CASE(N)                                                                          \
-    ffn_gather_kernel<WT, N><<<grid, kGatherThreads, 0, st>>>(Wg, Wu, Wd, hp, sp, c.d, c.group, c.k, \
-                                                              plan->partial)
+#define CS_GATHER_CASE(N)                                                                              \
+    ffn_gather_kernel<WT, N><<<grid, kGatherThreads, kRingBytes, st>>>(Wg, Wu, Wd, hp, sp, c.d, c.group, c.k, \
+                                                                       plan->partial)
         {
             StageTimer timer(plan, CS_STAGE_EXEC, st);
             if (cpt <= 1) CS_GATHER_CASE(1);
@@ -234,6 +287,17 @@ static cs_status gather_typed(cs_plan *plan, const cs_layer *L, const float *h, 
         plan->launches++;
         CS_CUDA_TRY(plan, cudaGetLastError());
     }
+    return CS_OK;
+}
+
+// The ring needs more dynamic shared memory than the default limit: opt in once per kernel.
+cs_status prepare_ffn_gather(cs_plan *plan) {
+#define CS_GATHER_ATTR(WT, N)                                                                       \
+    CS_CUDA_TRY(plan, cudaFuncSetAttribute(ffn_gather_kernel<WT, N>,                                \
+                                           cudaFuncAttributeMaxDynamicSharedMemorySize, kRingBytes))
+    CS_GATHER_ATTR(__nv_bfloat16, 1); CS_GATHER_ATTR(__nv_bfloat16, 2); CS_GATHER_ATTR(__nv_bfloat16, 4);
+    CS_GATHER_ATTR(float, 1); CS_GATHER_ATTR(float, 2); CS_GATHER_ATTR(float, 4);
+#undef CS_GATHER_ATTR
     return CS_OK;
 }
 
