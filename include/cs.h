@@ -111,6 +111,39 @@ cs_status cs_ffn_exec(cs_plan *plan, const cs_layer *layer, const float *h, cons
                       int32_t B, const float *residual, float *out, void *stream);
 
 /*
+ * cs_ffn_exec for callers that cannot allocate device memory.  (No counterpart in the paper: this
+ * is a deployment convenience of the library.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- inside a host framework that owns
+ * the whole device heap and forbids side allocations, in a process whose memory budget was fixed
+ * at start-up, or at a point where an allocation's implicit device synchronisation is not
+ * acceptable.  Such callers cannot create a cs_plan, because a plan's scratch comes from
+ * cudaMalloc.  This call needs no plan: the partial sums of the down projection are kept in an
+ * 8 MiB array that is compiled into the library (so every GPU that loads the library holds those
+ * 8 MiB until the process exits), and the call performs no cudaMalloc, cudaFree or any other
+ * allocating routine.
+ *
+ * Same mathematics, arguments and layouts as cs_ffn_exec (gather path), with the shape taken from
+ * `cfg` (d, d_ff, group, k, w_dtype are read; m, T, max_tokens, rms_eps are ignored).  Supports
+ * are not validated on the device: pass supports that are ascending, distinct and in [0, G), such
+ * as cs_recover writes.
+ *
+ * Limit: B * nx * d * 4 bytes must fit in the 8 MiB array, where nx >= ceil(k * group / 32) is the
+ * number of CTAs a token's rows are split over; e.g. d = 4096, k * group = 2816 allows B <= 5.
+ * Larger requests return CS_ERR_SHAPE and launch nothing.
+ *
+ * The first call on each device looks up the array's device address and raises the kernels'
+ * shared-memory limit; make that first call with the device current and before any stream
+ * capture begins.  All calls share the one array, which simply keeps whatever the last call
+ * left there (every call overwrites all it later reads, so nothing has to be cleared).  Two calls
+ * whose kernels can overlap on the GPU -- different streams, or different host threads on the
+ * same device -- would race on it: keep calls to this entry point ordered on one stream per device.
+ */
+cs_status cs_ffn_exec_static(const cs_config *cfg, const cs_layer *layer, const float *h,
+                             const int32_t *support, int32_t B, const float *residual, float *out,
+                             void *stream);
+
+/*
  * One decode step of one layer for B tokens with independent supports (Sec. 5; Sec. 12 online
  * phase):  n = rms_gamma ? RMSNorm(x) * rms_gamma : x;  y = S n;  (support, z) = recover(y);
  * x_out = (add_residual ? x : 0) + FFN(n, support).

@@ -69,6 +69,8 @@ def load_library():
     lib.cs_layer_step_host.argtypes = [vp, ctypes.POINTER(_Layer), vp, i32, vp, vp, vp]
     lib.cs_plan_enable_timing.argtypes = [vp, i32]
     lib.cs_plan_stage_times.argtypes = [vp, vp, ctypes.POINTER(f32 * 4)]
+    lib.cs_ffn_exec_static.argtypes = [ctypes.POINTER(_Config), ctypes.POINTER(_Layer), vp, vp, i32, vp, vp, vp]
+    lib.cs_ffn_exec_static.restype = ctypes.c_int
     lib.cs_last_device_status.argtypes = [vp, vp, ctypes.POINTER(i32)]
     lib.cs_launch_count.argtypes = [vp]
     lib.cs_launch_count.restype = ctypes.c_int64
@@ -205,6 +207,30 @@ def cs_ffn_exec(plan: Plan, layer: Layer, h, support, residual=None, out=None, s
                                     _ptr(support, torch.int32, "support", (B, plan.k)), B,
                                     _ptr(residual, torch.float32, "residual", (B, plan.d)),
                                     _ptr(out, torch.float32, "out", (B, plan.d)), _stream(stream)), "cs_ffn_exec")
+    return out
+
+
+def cs_ffn_exec_static(d: int, d_ff: int, group: int, k: int, layer: Layer, h, support, residual=None, out=None,
+                       stream=None):
+    """The gather FFN without a plan and without any device allocation by the library.
+
+    For callers that may not allocate on the device (see include/cs.h): the scratch is a fixed
+    8 MiB array inside the library.  ``out`` must be passed by such callers; it is only created
+    here, with torch, as a convenience for tests.  Raises CSError(CS_ERR_SHAPE) when B is too
+    large for the fixed array.
+    """
+    lib = load_library()
+    w_dtype = layer.tensors[2].dtype
+    code = {torch.float32: CS_F32, torch.bfloat16: CS_BF16}.get(w_dtype, -1)
+    cfg = _Config(d, d_ff, group, 1, k, 0, code, 1, 1e-5)
+    B = h.shape[0]
+    out = torch.empty((B, d), dtype=torch.float32, device=h.device) if out is None else out
+    st = lib.cs_ffn_exec_static(ctypes.byref(cfg), ctypes.byref(layer.c), _ptr(h, torch.float32, "h", (B, d)),
+                                _ptr(support, torch.int32, "support", (B, k)), B,
+                                _ptr(residual, torch.float32, "residual", (B, d)),
+                                _ptr(out, torch.float32, "out", (B, d)), _stream(stream))
+    if st != 0:
+        raise CSError(st, "cs_ffn_exec_static")
     return out
 
 

@@ -308,4 +308,94 @@ cs_status launch_ffn_gather(cs_plan *plan, const cs_layer *layer, const float *h
     return gather_typed<float>(plan, layer, h, support, B, residual, out, st);
 }
 
+
+// ---- cs_ffn_exec_static: the same gather FFN for callers that must not allocate ------------------
+//
+// The partial down-projections normally live in scratch a plan allocates with cudaMalloc.  This
+// entry point instead keeps them in the fixed array below, which is part of the library image: each
+// GPU that loads the library carries these 8 MiB until the process exits, and no call ever
+// allocates or frees anything.
+constexpr size_t kStaticScratchBytes = 8u << 20;
+static __device__ __align__(256) unsigned char g_static_partial[kStaticScratchBytes];
+
+constexpr int kStaticMaxDevices = 64;
+static float *g_static_ptr[kStaticMaxDevices];   // device address of g_static_partial, per device
+static int g_static_sms[kStaticMaxDevices];
+
+// Once per device, with that device current: look up where the array lives on the GPU (its name
+// in host code is only a handle, not an address a kernel could use) and opt the kernels in to the
+// shared-memory ring.  Neither call allocates.
+static cudaError_t static_setup(int dev) {
+    if (g_static_ptr[dev] != nullptr) return cudaSuccess;
+    void *p = nullptr;
+    cudaError_t e = cudaGetSymbolAddress(&p, g_static_partial);
+    if (e != cudaSuccess) return e;
+    int sms = 0;
+    e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return e;
+#define CS_STATIC_ATTR(WT, N)                                                                        \
+    if (e == cudaSuccess)                                                                            \
+        e = cudaFuncSetAttribute(ffn_gather_kernel<WT, N>, cudaFuncAttributeMaxDynamicSharedMemorySize, kRingBytes)
+    CS_STATIC_ATTR(__nv_bfloat16, 1); CS_STATIC_ATTR(__nv_bfloat16, 2); CS_STATIC_ATTR(__nv_bfloat16, 4);
+    CS_STATIC_ATTR(float, 1); CS_STATIC_ATTR(float, 2); CS_STATIC_ATTR(float, 4);
+#undef CS_STATIC_ATTR
+    if (e != cudaSuccess) return e;
+    g_static_sms[dev] = sms;
+    g_static_ptr[dev] = static_cast<float *>(p);
+    return cudaSuccess;
+}
+
+template <typename WT>
+static cudaError_t static_launch(const cs_config &c, const cs_layer *L, const float *h, const int32_t *support,
+                                 int B, int nx, float *partial, const float *residual, float *out,
+                                 cudaStream_t st) {
+    constexpr int E = Chunk<WT>::kElems;
+    const int cpt = (c.d / E + kGatherThreads - 1) / kGatherThreads;
+    const WT *Wg = static_cast<const WT *>(L->W_gate), *Wu = static_cast<const WT *>(L->W_up),
+             *Wd = static_cast<const WT *>(L->Wd_t);
+    dim3 grid(nx, B);
+    if (cpt <= 1)
+        ffn_gather_kernel<WT, 1><<<grid, kGatherThreads, kRingBytes, st>>>(Wg, Wu, Wd, h, support, c.d, c.group, c.k, partial);
+    else if (cpt <= 2)
+        ffn_gather_kernel<WT, 2><<<grid, kGatherThreads, kRingBytes, st>>>(Wg, Wu, Wd, h, support, c.d, c.group, c.k, partial);
+    else
+        ffn_gather_kernel<WT, 4><<<grid, kGatherThreads, kRingBytes, st>>>(Wg, Wu, Wd, h, support, c.d, c.group, c.k, partial);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    dim3 rgrid((c.d / 4 + 31) / 32, B);
+    reduce_partials_kernel<<<rgrid, 32 * kReduceGroups, 0, st>>>(partial, nx, c.d, residual, out);
+    return cudaGetLastError();
+}
+
 }  // namespace cs
+
+extern "C" cs_status cs_ffn_exec_static(const cs_config *cfg, const cs_layer *layer, const float *h,
+                                        const int32_t *support, int32_t B, const float *residual, float *out,
+                                        void *stream) {
+    using namespace cs;
+    if (cfg == nullptr || layer == nullptr || h == nullptr || support == nullptr || out == nullptr) return CS_ERR_NULL;
+    if (layer->W_gate == nullptr || layer->W_up == nullptr || layer->Wd_t == nullptr) return CS_ERR_NULL;
+    if (cfg->d <= 0 || cfg->group <= 0 || cfg->k <= 0 || cfg->d_ff <= 0 || cfg->d_ff % cfg->group != 0 ||
+        cfg->k > cfg->d_ff / cfg->group || B <= 0)
+        return CS_ERR_SHAPE;
+    if ((cfg->group != 64 && cfg->group != 128) || cfg->d > kMaxD || cfg->d % 64 != 0 ||
+        cfg->d_ff / cfg->group > kMaxG || (cfg->w_dtype != CS_F32 && cfg->w_dtype != CS_BF16))
+        return CS_ERR_UNSUPPORTED;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kStaticMaxDevices) return CS_ERR_CUDA;
+    if (static_setup(dev) != cudaSuccess) return CS_ERR_CUDA;
+    // B * nx partial vectors of d floats must fit the fixed array; nx may shrink down to the point
+    // where a CTA would own more than kGatherMaxRows rows, beyond that the request is too large.
+    const int rows_total = cfg->k * cfg->group;
+    const int nx_min = (rows_total + kGatherMaxRows - 1) / kGatherMaxRows;
+    const size_t per_vec = (size_t)cfg->d * sizeof(float);
+    const size_t fit = kStaticScratchBytes / (per_vec * (size_t)B);
+    if (fit < (size_t)nx_min) return CS_ERR_SHAPE;
+    int nx = max(g_static_sms[dev] / B, nx_min);
+    nx = (int)min((size_t)min(nx, rows_total), fit);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaError_t e = cfg->w_dtype == CS_BF16
+        ? static_launch<__nv_bfloat16>(*cfg, layer, h, support, B, nx, g_static_ptr[dev], residual, out, st)
+        : static_launch<float>(*cfg, layer, h, support, B, nx, g_static_ptr[dev], residual, out, st);
+    return e == cudaSuccess ? CS_OK : CS_ERR_CUDA;
+}
