@@ -5,15 +5,19 @@
 //     a[c]      = silu(W_gate[c,:] . h) * (W_up[c,:] . h)
 //     partial[:] = sum_c a[c] * Wd_t[c,:]
 // so gate, up and down rows of a channel are consumed by the same CTA and nothing but the
-// d-vector of partial sums crosses CTAs.  Inside a CTA the hidden dimension is split over all
-// threads: thread i owns 16-byte chunk i (+512, ...) of every row.
+// d-vector of partial sums crosses CTAs.
 //
-// The kernel is a pure HBM stream (3 * rows * d weight elements, each used once), so what matters
-// is bytes in flight.  Every thread runs its own cp.async ring: it copies its 16-byte chunks of
-// the next rows into its private slots of a shared-memory ring (L2 -> shared, bypassing L1 and
-// registers), up to kRingBytes per CTA ahead of use, and reads back only what it copied itself,
-// so the ring needs no barrier at all.  The down rows are already in flight while the gate/up
-// results are being folded across warps.
+// The kernel is a pure HBM stream (3 * rows * d weight elements, each used once), so two things
+// matter: bytes in flight, and few instructions per byte.
+//   - Every lane copies its own 16-byte chunks with cp.async (L2 -> shared, bypassing L1 and
+//     registers) into slots only it reads back, so the rings need no barrier: each warp keeps
+//     kWarpRing bytes in flight, kRingBytes per CTA.
+//   - Gate/up phase: a warp takes (row, segment) units, a segment being kUnitChunks chunks per lane
+//     of the gate row and of the up row; the two warp reductions per unit are amortised over
+//     2 * kUnitChunks chunks per lane.  Segment partials are kept apart and added in segment order.
+//   - Down phase: thread i owns chunk i (+512, ...) of every row, so the partial output stays in
+//     registers; the down rows are copied into the warp's ring as soon as the warp has finished
+//     its gate/up units, i.e. they are in flight while the activations are being folded.
 // The partial d-vectors are summed in a fixed order by reduce_partials_kernel (deterministic,
 // no atomics), which also adds the residual.
 #include "cs_internal.cuh"
@@ -22,8 +26,14 @@ namespace cs {
 
 __device__ __forceinline__ float silu(float x) { return x / (1.f + __expf(-x)); }
 
+constexpr int kGatherWarps = kGatherThreads / 32;
 constexpr int kRingBytes = 192 * 1024;
-constexpr int kItemBytes = 2 * 16 * kGatherThreads;  // two rows' worth of one chunk per thread
+constexpr int kWarpRing = kRingBytes / kGatherWarps;       // 12 KB per warp
+constexpr int kUnitChunks = 4;                             // chunks per lane, matrix and unit
+constexpr int kUnitBytes = 2 * kUnitChunks * 32 * 16;      // gate + up: 4 KB
+constexpr int kUnitStages = kWarpRing / kUnitBytes;        // 3 units in flight per warp
+constexpr int kLaneSlots = kWarpRing / (32 * 16);          // 24 chunks per lane in the down phase
+constexpr int kMaxSegs = kMaxD * 4 / (kUnitChunks * 32 * 16);  // 16 (f32 rows of 8192)
 
 __device__ __forceinline__ void cp_async16(void *smem_dst, const void *gmem_src) {
     const uint32_t s = static_cast<uint32_t>(__cvta_generic_to_shared(smem_dst));
@@ -34,19 +44,19 @@ template <int N> __device__ __forceinline__ void cp_async_wait() {
     asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
 }
 
-// CPT = 16-byte chunks per thread and row.  Ring item i: i < nrows -> (gate row i, up row i);
-// i >= nrows -> (down row 2(i-nrows), down row 2(i-nrows)+1).
-template <typename WT, int CPT>
-__global__ void __launch_bounds__(kGatherThreads)
+// CPT = 16-byte chunks per thread and row in the down phase (row bytes / (512 * 16), rounded up).
+// FULL = every row is a whole number of units and of 512-chunk slices: no bounds checks inside.
+template <typename WT, int CPT, bool FULL>
+__global__ void __launch_bounds__(kGatherThreads, 1)
 ffn_gather_kernel(const WT *__restrict__ Wg, const WT *__restrict__ Wu, const WT *__restrict__ Wdt,
                   const float *__restrict__ h, const int32_t *__restrict__ support, int d, int b, int k,
                   float *__restrict__ partial) {
     constexpr int E = Chunk<WT>::kElems;
-    constexpr int kWarps = kGatherThreads / 32;
-    constexpr int NS = kRingBytes / (kItemBytes * CPT);  // ring stages
-    extern __shared__ __align__(16) uint4 ring[];        // [NS][2][CPT][kGatherThreads]
-    __shared__ float red[2 * kGatherMaxRows][kWarps];
-    __shared__ float a_s[kGatherMaxRows + 1];
+    constexpr int DR = kLaneSlots / CPT;               // down rows in flight per thread
+    constexpr int kSegElems = kUnitChunks * 32 * E;    // elements of one row segment
+    extern __shared__ __align__(16) uint4 ring[];      // [kGatherWarps][kWarpRing / 16]
+    __shared__ float red[kGatherMaxRows][kMaxSegs][2];
+    __shared__ float a_s[kGatherMaxRows];
     __shared__ int chan_s[kGatherMaxRows];
 
     const int t = blockIdx.y, nx = gridDim.x;
@@ -54,130 +64,134 @@ ffn_gather_kernel(const WT *__restrict__ Wg, const WT *__restrict__ Wu, const WT
     const int r_begin = (int)(((long long)rows_total * blockIdx.x) / nx);
     const int r_end = (int)(((long long)rows_total * (blockIdx.x + 1)) / nx);
     const int nrows = r_end - r_begin;
-    const int nitems = nrows + (nrows + 1) / 2;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int chunks = d / E;
+    const int chunks = d / E;                                       // chunks per row
+    const int nseg = (chunks + kUnitChunks * 32 - 1) / (kUnitChunks * 32);
+    const int nunits = nrows * nseg;
 
     if (tid < nrows) {
         const int c = r_begin + tid;
         chan_s[tid] = support[(size_t)t * k + c / b] * b + c % b;
     }
-    if (tid == 0) a_s[nrows] = 0.f;  // pad for an odd last down pair
     __syncthreads();
 
-    auto slot = [&](int stage, int half, int j) -> uint4 * {
-        return ring + (((size_t)stage * 2 + half) * CPT + j) * kGatherThreads + tid;
+    uint4 *wring = ring + (size_t)warp * (kWarpRing / 16) + lane;   // this lane's column of the warp ring
+    // ---- gate / up: units u = warp, warp + 16, ... ; unit u = (row u / nseg, segment u % nseg).
+    // Two cursors (copy issue, consumption) walk the units incrementally: no division in the loop.
+    const int step_r = kGatherWarps / nseg, step_s = kGatherWarps % nseg;
+    struct Cursor { int u, r, seg; };
+    auto advance = [&](Cursor &c) {
+        c.u += kGatherWarps; c.r += step_r; c.seg += step_s;
+        if (c.seg >= nseg) { c.seg -= nseg; ++c.r; }
     };
-    auto issue = [&](int i) {
-        if (i < nitems) {
-            const WT *p0, *p1;
-            bool two = true;
-            if (i < nrows) {
-                const size_t base = (size_t)chan_s[i] * d;
-                p0 = Wg + base; p1 = Wu + base;
-            } else {
-                const int r = 2 * (i - nrows);
-                two = r + 1 < nrows;
-                p0 = Wdt + (size_t)chan_s[r] * d;
-                p1 = Wdt + (size_t)chan_s[two ? r + 1 : r] * d;
-            }
-            const int stage = i % NS;
+    Cursor ci{warp, warp / nseg, warp % nseg}, cc = ci;
+    const WT *wg_lane = Wg + lane * E, *wu_lane = Wu + lane * E;
+    const float *h_lane = h + (size_t)t * d + lane * E;
+
+    auto issue_unit = [&](int stage) {
+        if (ci.u < nunits) {
+            const size_t off = (size_t)chan_s[ci.r] * d + (size_t)ci.seg * kSegElems;
+            const WT *pg = wg_lane + off, *pu = wu_lane + off;
+            uint4 *dst = wring + stage * (2 * kUnitChunks * 32);
 #pragma unroll
-            for (int j = 0; j < CPT; ++j) {
-                const int c = tid + j * kGatherThreads;
-                if (c < chunks) {
-                    cp_async16(slot(stage, 0, j), p0 + (size_t)c * E);
-                    if (two) cp_async16(slot(stage, 1, j), p1 + (size_t)c * E);
+            for (int j = 0; j < kUnitChunks; ++j) {
+                if (FULL || (ci.seg * kUnitChunks + j) * 32 + lane < chunks) {
+                    cp_async16(dst + j * 32, pg + j * 32 * E);
+                    cp_async16(dst + (kUnitChunks + j) * 32, pu + j * 32 * E);
                 }
             }
         }
-        cp_async_commit();  // one group per item, empty past the end, so the wait count stays fixed
+        cp_async_commit();  // one group per unit, empty past the end, so the wait count stays fixed
+        advance(ci);
     };
+#pragma unroll
+    for (int i = 0; i < kUnitStages; ++i) issue_unit(i);
+    int stage = 0;
 #pragma unroll 1
-    for (int i = 0; i < NS; ++i) issue(i);
-
-    // this thread's slice of h
-    float hv[CPT][E];
+    for (; cc.u < nunits; advance(cc)) {
+        cp_async_wait<kUnitStages - 1>();
+        const uint4 *src = wring + stage * (2 * kUnitChunks * 32);
+        const float *hp = h_lane + cc.seg * kSegElems;
+        float g = 0.f, up = 0.f;
 #pragma unroll
-    for (int j = 0; j < CPT; ++j) {
-        const int c = tid + j * kGatherThreads;
+        for (int j = 0; j < kUnitChunks; ++j) {
+            if (FULL || (cc.seg * kUnitChunks + j) * 32 + lane < chunks) {
+                float hv[E], wg[E], wu[E];
 #pragma unroll
-        for (int e = 0; e < E; e += 4) {
-            float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (c < chunks) v = *reinterpret_cast<const float4 *>(h + (size_t)t * d + (size_t)c * E + e);
-            hv[j][e] = v.x; hv[j][e + 1] = v.y; hv[j][e + 2] = v.z; hv[j][e + 3] = v.w;
-        }
-    }
-
-    // ---- gate / up rows
-#pragma unroll 1
-    for (int i = 0; i < nrows; ++i) {
-        cp_async_wait<NS - 1>();
-        const int stage = i % NS;
-        float g = 0.f, u = 0.f;
+                for (int e = 0; e < E; e += 4) {
+                    const float4 v = __ldg(reinterpret_cast<const float4 *>(hp + j * 32 * E + e));
+                    hv[e] = v.x; hv[e + 1] = v.y; hv[e + 2] = v.z; hv[e + 3] = v.w;
+                }
+                Chunk<WT>::widen(src[j * 32], wg);
+                Chunk<WT>::widen(src[(kUnitChunks + j) * 32], wu);
 #pragma unroll
-        for (int j = 0; j < CPT; ++j) {
-            const int c = tid + j * kGatherThreads;
-            if (c < chunks) {
-                float wg[E], wu[E];
-                Chunk<WT>::widen(*slot(stage, 0, j), wg);
-                Chunk<WT>::widen(*slot(stage, 1, j), wu);
-#pragma unroll
-                for (int e = 0; e < E; ++e) { g = fmaf(wg[e], hv[j][e], g); u = fmaf(wu[e], hv[j][e], u); }
+                for (int e = 0; e < E; ++e) { g = fmaf(wg[e], hv[e], g); up = fmaf(wu[e], hv[e], up); }
             }
         }
-        issue(i + NS);  // refill the slot just consumed (after its values were used above)
-        g = warp_sum(g); u = warp_sum(u);
-        if (lane == 0) { red[2 * i][warp] = g; red[2 * i + 1][warp] = u; }
+        issue_unit(stage);  // refill the stage just consumed (its values were used above)
+        stage = stage + 1 == kUnitStages ? 0 : stage + 1;
+        g = warp_sum(g); up = warp_sum(up);
+        if (lane == 0) { red[cc.r][cc.seg][0] = g; red[cc.r][cc.seg][1] = up; }
     }
+    cp_async_wait<0>();
+
+    // ---- down rows: thread i owns chunks i, i + 512, ... of every row; lane slots of the warp ring
+    const WT *wd_thread = Wdt + tid * E;
+    int issue_r = 0, issue_stage = 0;
+    auto issue_down = [&]() {
+        if (issue_r < nrows) {
+            const WT *p = wd_thread + (size_t)chan_s[issue_r] * d;
+            uint4 *dst = wring + issue_stage * (CPT * 32);
+#pragma unroll
+            for (int j = 0; j < CPT; ++j)
+                if (FULL || tid + j * kGatherThreads < chunks) cp_async16(dst + j * 32, p + j * kGatherThreads * E);
+        }
+        cp_async_commit();
+        ++issue_r;
+        issue_stage = issue_stage + 1 == DR ? 0 : issue_stage + 1;
+    };
+#pragma unroll 1
+    for (int r = 0; r < DR; ++r) issue_down();
+
     __syncthreads();
     if (tid < nrows) {
-        float g = 0.f, u = 0.f;
-#pragma unroll
-        for (int w = 0; w < kWarps; ++w) { g += red[2 * tid][w]; u += red[2 * tid + 1][w]; }
-        a_s[tid] = silu(g) * u;
+        float g = 0.f, up = 0.f;
+        for (int sgm = 0; sgm < nseg; ++sgm) { g += red[tid][sgm][0]; up += red[tid][sgm][1]; }
+        a_s[tid] = silu(g) * up;
     }
     __syncthreads();
 
-    // ---- down rows, two per ring item
     float acc[CPT][E];
 #pragma unroll
     for (int j = 0; j < CPT; ++j)
 #pragma unroll
         for (int e = 0; e < E; ++e) acc[j][e] = 0.f;
+    stage = 0;
 #pragma unroll 1
-    for (int i = nrows; i < nitems; ++i) {
-        cp_async_wait<NS - 1>();
-        const int stage = i % NS;
-        const int r = 2 * (i - nrows);
-        const float a0 = a_s[r], a1 = a_s[r + 1];
-        const bool two = r + 1 < nrows;
+    for (int r = 0; r < nrows; ++r) {
+        cp_async_wait<DR - 1>();
+        const uint4 *src = wring + stage * (CPT * 32);
+        const float a = a_s[r];
 #pragma unroll
         for (int j = 0; j < CPT; ++j) {
-            const int c = tid + j * kGatherThreads;
-            if (c < chunks) {
-                float w0[E], w1[E];
-                Chunk<WT>::widen(*slot(stage, 0, j), w0);
+            if (FULL || tid + j * kGatherThreads < chunks) {
+                float w[E];
+                Chunk<WT>::widen(src[j * 32], w);
 #pragma unroll
-                for (int e = 0; e < E; ++e) acc[j][e] = fmaf(a0, w0[e], acc[j][e]);
-                if (two) {
-                    Chunk<WT>::widen(*slot(stage, 1, j), w1);
-#pragma unroll
-                    for (int e = 0; e < E; ++e) acc[j][e] = fmaf(a1, w1[e], acc[j][e]);
-                }
+                for (int e = 0; e < E; ++e) acc[j][e] = fmaf(a, w[e], acc[j][e]);
             }
         }
-        issue(i + NS);
+        issue_down();
+        stage = stage + 1 == DR ? 0 : stage + 1;
     }
     cp_async_wait<0>();
-    float *dst = partial + ((size_t)t * nx + blockIdx.x) * d;
+    float *dst = partial + ((size_t)t * nx + blockIdx.x) * d + tid * E;
 #pragma unroll
     for (int j = 0; j < CPT; ++j) {
-        const int c = tid + j * kGatherThreads;
-        if (c < chunks) {
+        if (FULL || tid + j * kGatherThreads < chunks) {
 #pragma unroll
             for (int e = 0; e < E; e += 4)
-                *reinterpret_cast<float4 *>(dst + (size_t)c * E + e) =
+                *reinterpret_cast<float4 *>(dst + j * kGatherThreads * E + e) =
                     make_float4(acc[j][e], acc[j][e + 1], acc[j][e + 2], acc[j][e + 3]);
         }
     }
@@ -249,6 +263,20 @@ cs_status launch_check_support(cs_plan *plan, const int32_t *support, int B, cud
     return CS_OK;
 }
 
+// Picks the instantiation: chunks per thread in the down phase, and whether rows need bounds checks.
+template <typename WT>
+static void launch_gather_kernel(dim3 grid, cudaStream_t st, int cpt, int chunks, const WT *Wg, const WT *Wu,
+                                 const WT *Wd, const float *h, const int32_t *sup, int d, int b, int k,
+                                 float *partial) {
+    const bool full = chunks % kGatherThreads == 0 && (cpt == 1 || cpt == 2 || cpt == 4);
+#define CS_GATHER_CASE(N, F)                                                                          \
+    ffn_gather_kernel<WT, N, F><<<grid, kGatherThreads, kRingBytes, st>>>(Wg, Wu, Wd, h, sup, d, b, k, partial)
+    if (cpt <= 1) { if (full) CS_GATHER_CASE(1, true); else CS_GATHER_CASE(1, false); }
+    else if (cpt <= 2) { if (full) CS_GATHER_CASE(2, true); else CS_GATHER_CASE(2, false); }
+    else { if (full) CS_GATHER_CASE(4, true); else CS_GATHER_CASE(4, false); }
+#undef CS_GATHER_CASE
+}
+
 template <typename WT>
 static cs_status gather_typed(cs_plan *plan, const cs_layer *L, const float *h, const int32_t *support,
                               int B, const float *residual, float *out, cudaStream_t st) {
@@ -266,16 +294,10 @@ static cs_status gather_typed(cs_plan *plan, const cs_layer *L, const float *h, 
         dim3 grid(nx, nb);
         const float *hp = h + (size_t)t0 * c.d;
         const int32_t *sp = support + (size_t)t0 * c.k;
-#define CS_GATHER_CASE(N)                                                                              \
-    ffn_gather_kernel<WT, N><<<grid, kGatherThreads, kRingBytes, st>>>(Wg, Wu, Wd, hp, sp, c.d, c.group, c.k, \
-                                                                       plan->partial)
         {
             StageTimer timer(plan, CS_STAGE_EXEC, st);
-            if (cpt <= 1) CS_GATHER_CASE(1);
-            else if (cpt <= 2) CS_GATHER_CASE(2);
-            else CS_GATHER_CASE(4);
+            launch_gather_kernel<WT>(grid, st, cpt, c.d / E, Wg, Wu, Wd, hp, sp, c.d, c.group, c.k, plan->partial);
         }
-#undef CS_GATHER_CASE
         plan->launches++;
         CS_CUDA_TRY(plan, cudaGetLastError());
         dim3 rgrid((c.d / 4 + 31) / 32, nb);
@@ -293,7 +315,9 @@ static cs_status gather_typed(cs_plan *plan, const cs_layer *L, const float *h, 
 // The ring needs more dynamic shared memory than the default limit: opt in once per kernel.
 cs_status prepare_ffn_gather(cs_plan *plan) {
 #define CS_GATHER_ATTR(WT, N)                                                                       \
-    CS_CUDA_TRY(plan, cudaFuncSetAttribute(ffn_gather_kernel<WT, N>,                                \
+    CS_CUDA_TRY(plan, cudaFuncSetAttribute(ffn_gather_kernel<WT, N, true>,                          \
+                                           cudaFuncAttributeMaxDynamicSharedMemorySize, kRingBytes)); \
+    CS_CUDA_TRY(plan, cudaFuncSetAttribute(ffn_gather_kernel<WT, N, false>,                         \
                                            cudaFuncAttributeMaxDynamicSharedMemorySize, kRingBytes))
     CS_GATHER_ATTR(__nv_bfloat16, 1); CS_GATHER_ATTR(__nv_bfloat16, 2); CS_GATHER_ATTR(__nv_bfloat16, 4);
     CS_GATHER_ATTR(float, 1); CS_GATHER_ATTR(float, 2); CS_GATHER_ATTR(float, 4);
@@ -335,7 +359,9 @@ static cudaError_t static_setup(int dev) {
     if (e != cudaSuccess) return e;
 #define CS_STATIC_ATTR(WT, N)                                                                        \
     if (e == cudaSuccess)                                                                            \
-        e = cudaFuncSetAttribute(ffn_gather_kernel<WT, N>, cudaFuncAttributeMaxDynamicSharedMemorySize, kRingBytes)
+        e = cudaFuncSetAttribute(ffn_gather_kernel<WT, N, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kRingBytes); \
+    if (e == cudaSuccess)                                                                            \
+        e = cudaFuncSetAttribute(ffn_gather_kernel<WT, N, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kRingBytes)
     CS_STATIC_ATTR(__nv_bfloat16, 1); CS_STATIC_ATTR(__nv_bfloat16, 2); CS_STATIC_ATTR(__nv_bfloat16, 4);
     CS_STATIC_ATTR(float, 1); CS_STATIC_ATTR(float, 2); CS_STATIC_ATTR(float, 4);
 #undef CS_STATIC_ATTR
@@ -354,12 +380,7 @@ static cudaError_t static_launch(const cs_config &c, const cs_layer *L, const fl
     const WT *Wg = static_cast<const WT *>(L->W_gate), *Wu = static_cast<const WT *>(L->W_up),
              *Wd = static_cast<const WT *>(L->Wd_t);
     dim3 grid(nx, B);
-    if (cpt <= 1)
-        ffn_gather_kernel<WT, 1><<<grid, kGatherThreads, kRingBytes, st>>>(Wg, Wu, Wd, h, support, c.d, c.group, c.k, partial);
-    else if (cpt <= 2)
-        ffn_gather_kernel<WT, 2><<<grid, kGatherThreads, kRingBytes, st>>>(Wg, Wu, Wd, h, support, c.d, c.group, c.k, partial);
-    else
-        ffn_gather_kernel<WT, 4><<<grid, kGatherThreads, kRingBytes, st>>>(Wg, Wu, Wd, h, support, c.d, c.group, c.k, partial);
+    launch_gather_kernel<WT>(grid, st, cpt, c.d / E, Wg, Wu, Wd, h, support, c.d, c.group, c.k, partial);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     dim3 rgrid((c.d / 4 + 31) / 32, B);
