@@ -105,10 +105,23 @@ cs_status cs_recover(cs_plan *plan, const float *Phi, float mu, const float *y, 
  *   in [0,G); residual [B,d] f32 or NULL; out [B,d] f32.  out may alias residual, not h.
  * layer->S, Phi, rms_gamma, mu and add_residual are ignored.  Small batches run as a gather GEMV
  * that streams each token's active rows once; large batches bucket tokens by group and run the
- * active blocks on the tensor cores (activations rounded to bf16 there).
+ * active blocks on the tensor cores; f32 activations enter those GEMMs as two bf16 parts (value and
+ * remainder), which keeps the result at f32-level accuracy.
  */
 cs_status cs_ffn_exec(cs_plan *plan, const cs_layer *layer, const float *h, const int32_t *support,
                       int32_t B, const float *residual, float *out, void *stream);
+
+/*
+ * Dispatch step between estimator and actuator (Sec. 7: the estimator's output selects which
+ * precompiled execution path runs, here which tokens each group's weight block serves): inverts
+ * token -> groups into group -> tokens.
+ *   support [B,k] int32 ascending  ->  counts [G] (tokens per group), offsets [G+1] (exclusive
+ *   prefix sums), token_ids [B*k] (the tokens of group g, ascending, at offsets[g] .. offsets[g+1]).
+ * cs_ffn_exec runs this itself for large batches; the call exists for callers that want the
+ * buckets (support diversity statistics, their own scheduling).
+ */
+cs_status cs_bucket(cs_plan *plan, const int32_t *support, int32_t B, int32_t *counts, int32_t *offsets,
+                    int32_t *token_ids, void *stream);
 
 /*
  * cs_ffn_exec for callers that cannot allocate device memory.  (No counterpart in the paper: this

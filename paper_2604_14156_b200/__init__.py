@@ -6,6 +6,6 @@ CUDA kernels under ``csrc/``.  There is no CPU implementation: loading fails lou
 shared library is missing and calls fail on non-CUDA tensors.
 """
 from .binding import (  # noqa: F401
-    CSError, Layer, Plan, cs_ffn_exec, cs_ffn_exec_shared, cs_ffn_exec_static, cs_layer_step, cs_layer_step_host, cs_prompt_support,
+    CSError, Layer, Plan, cs_bucket, cs_ffn_exec, cs_ffn_exec_shared, cs_ffn_exec_static, cs_layer_step, cs_layer_step_host, cs_prompt_support,
     cs_recover, cs_sketch, exported_symbols, library_path, load_library,
 )

@@ -71,6 +71,8 @@ def load_library():
     lib.cs_plan_stage_times.argtypes = [vp, vp, ctypes.POINTER(f32 * 4)]
     lib.cs_ffn_exec_static.argtypes = [ctypes.POINTER(_Config), ctypes.POINTER(_Layer), vp, vp, i32, vp, vp, vp]
     lib.cs_ffn_exec_static.restype = ctypes.c_int
+    lib.cs_bucket.argtypes = [vp, vp, i32, vp, vp, vp, vp]
+    lib.cs_bucket.restype = ctypes.c_int
     lib.cs_last_device_status.argtypes = [vp, vp, ctypes.POINTER(i32)]
     lib.cs_launch_count.argtypes = [vp]
     lib.cs_launch_count.restype = ctypes.c_int64
@@ -232,6 +234,19 @@ def cs_ffn_exec_static(d: int, d_ff: int, group: int, k: int, layer: Layer, h, s
     if st != 0:
         raise CSError(st, "cs_ffn_exec_static")
     return out
+
+
+def cs_bucket(plan: Plan, support, stream=None):
+    """(counts [G], offsets [G+1], token_ids [B*k]) of the group -> tokens inversion."""
+    B = support.shape[0]
+    dev = support.device
+    counts = torch.empty((plan.G,), dtype=torch.int32, device=dev)
+    offsets = torch.empty((plan.G + 1,), dtype=torch.int32, device=dev)
+    token_ids = torch.empty((B * plan.k,), dtype=torch.int32, device=dev)
+    plan.check(plan.lib.cs_bucket(plan.handle, _ptr(support, torch.int32, "support", (B, plan.k)), B,
+                                  counts.data_ptr(), offsets.data_ptr(), token_ids.data_ptr(), _stream(stream)),
+               "cs_bucket")
+    return counts, offsets, token_ids
 
 
 def cs_layer_step(plan: Plan, layer: Layer, x, x_out=None, want_aux: bool = True, stream=None):

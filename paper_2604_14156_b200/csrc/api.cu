@@ -62,12 +62,29 @@ cs_status cs_plan_create(const cs_config *cfg, cs_plan **out) {
     alloc((void **)&p->hbar, (size_t)cfg->d * sizeof(float));
     alloc((void **)&p->colsum, (size_t)p->mean_row_blocks * cfg->d * sizeof(float));
     alloc((void **)&p->status, sizeof(DeviceStatus));
+    p->mma_ok = cfg->w_dtype == CS_BF16 && cfg->group == 128 && cfg->d % 256 == 0;
+    alloc((void **)&p->mask, nt * 4 * sizeof(uint32_t));
+    alloc((void **)&p->counts, (size_t)kMaxG * sizeof(int32_t));
+    alloc((void **)&p->offsets, (size_t)(kMaxG + 1) * sizeof(int32_t));
+    alloc((void **)&p->token_ids, nt * cfg->k * sizeof(int32_t));
+    alloc((void **)&p->glist, (size_t)kMaxG * sizeof(int32_t));
+    alloc((void **)&p->nu, sizeof(int32_t));
+    if (p->mma_ok) {
+        const size_t m_pad = (nt + 127) / 128 * 128;
+        p->mma_slices = max(1, min(16, p->sm_count / max(1, cfg->d / 256)));
+        alloc((void **)&p->x_bf16, 2 * nt * cfg->d * 2);
+        alloc((void **)&p->act, 2 * nt * cfg->d_ff * 2);
+        // slices * padded tokens never exceeds 128 * (SMs / column tiles): see launch_ffn_mma
+        const size_t slice_rows = (size_t)128 * (p->sm_count / max(1, cfg->d / 256) + 1);
+        alloc((void **)&p->mma_partial, max(slice_rows, m_pad) * cfg->d * sizeof(float));
+    }
     alloc((void **)&p->x_host_in, nt * cfg->d * sizeof(float));
     alloc((void **)&p->x_host_out, nt * cfg->d * sizeof(float));
     for (int i = 0; i < 2 * CS_STAGE_COUNT; ++i)
         if (e == cudaSuccess) e = cudaEventCreate(&p->ev[i]);
     if (e == cudaSuccess) e = cudaMemset(p->status, 0, sizeof(DeviceStatus));
     if (e == cudaSuccess && prepare_ffn_gather(p) != CS_OK) e = cudaErrorUnknown;
+    if (e == cudaSuccess && p->mma_ok && prepare_ffn_mma(p) != CS_OK) e = cudaErrorUnknown;
     if (e != cudaSuccess) {
         cs_plan_destroy(p);
         return CS_ERR_CUDA;
@@ -81,6 +98,8 @@ cs_status cs_plan_destroy(cs_plan *p) {
     cudaFree(p->n_buf); cudaFree(p->y_buf); cudaFree(p->sup_buf); cudaFree(p->z_buf);
     cudaFree(p->resid_buf); cudaFree(p->partial); cudaFree(p->hbar); cudaFree(p->colsum);
     cudaFree(p->status); cudaFree(p->x_host_in); cudaFree(p->x_host_out);
+    cudaFree(p->mask); cudaFree(p->counts); cudaFree(p->offsets); cudaFree(p->token_ids); cudaFree(p->glist);
+    cudaFree(p->nu); cudaFree(p->x_bf16); cudaFree(p->act); cudaFree(p->mma_partial);
     for (int i = 0; i < 2 * CS_STAGE_COUNT; ++i)
         if (p->ev[i] != nullptr) cudaEventDestroy(p->ev[i]);
     delete p;
@@ -108,6 +127,21 @@ static cs_status check_weights(const cs_layer *L) {
     return CS_OK;
 }
 
+// Large decode batches on the tensor cores: activations to bf16, buckets / masks / union list from
+// the supports, then the two grouped GEMMs over the union.
+static cs_status exec_dispatch(cs_plan *plan, const cs_layer *layer, const float *h, const int32_t *support,
+                               int B, const float *residual, float *out, cudaStream_t st) {
+    if (!plan->mma_ok || B < kMmaMinTokens) return launch_ffn_gather(plan, layer, h, support, B, residual, out, st);
+    // f32 activations go in as two bf16 parts so that the result keeps f32-level accuracy
+    __nv_bfloat16 *x_hi = static_cast<__nv_bfloat16 *>(plan->x_bf16);
+    __nv_bfloat16 *x_lo = x_hi + (size_t)plan->cfg.max_tokens * plan->cfg.d;
+    cs_status s = launch_split_bf16(plan, h, x_hi, x_lo, (size_t)B * plan->cfg.d, st);
+    if (s != CS_OK) return s;
+    s = launch_bucket(plan, support, B, st);
+    if (s != CS_OK) return s;
+    return launch_ffn_mma(plan, layer, x_hi, x_lo, B, plan->glist, plan->nu, 0, plan->mask, residual, out, nullptr, st);
+}
+
 cs_status cs_ffn_exec(cs_plan *plan, const cs_layer *layer, const float *h, const int32_t *support,
                       int32_t B, const float *residual, float *out, void *stream) {
     if (plan == nullptr || h == nullptr || support == nullptr || out == nullptr) return CS_ERR_NULL;
@@ -118,7 +152,18 @@ cs_status cs_ffn_exec(cs_plan *plan, const cs_layer *layer, const float *h, cons
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     s = launch_check_support(plan, support, B, st);
     if (s != CS_OK) return s;
-    return launch_ffn_gather(plan, layer, h, support, B, residual, out, st);
+    return exec_dispatch(plan, layer, h, support, B, residual, out, st);
+}
+
+cs_status cs_bucket(cs_plan *plan, const int32_t *support, int32_t B, int32_t *counts, int32_t *offsets,
+                    int32_t *token_ids, void *stream) {
+    if (plan == nullptr || support == nullptr || counts == nullptr || offsets == nullptr || token_ids == nullptr)
+        return CS_ERR_NULL;
+    if (B <= 0 || B > plan->cfg.max_tokens) return CS_ERR_SHAPE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cs_status s = launch_check_support(plan, support, B, st);
+    if (s != CS_OK) return s;
+    return launch_bucket(plan, support, B, st, counts, offsets, token_ids);
 }
 
 cs_status cs_layer_step(cs_plan *plan, const cs_layer *layer, const float *x, int32_t B, float *x_out,
@@ -141,7 +186,7 @@ cs_status cs_layer_step(cs_plan *plan, const cs_layer *layer, const float *x, in
     s = launch_recover(plan, layer->Phi, layer->mu, plan->y_buf, B, sup, z_out, resid_out, st);
     if (s != CS_OK) return s;
     // supports produced by cs_recover are valid by construction: no device check here
-    return launch_ffn_gather(plan, layer, n, sup, B, layer->add_residual ? x : nullptr, x_out, st);
+    return exec_dispatch(plan, layer, n, sup, B, layer->add_residual ? x : nullptr, x_out, st);
 }
 
 cs_status cs_layer_step_host(cs_plan *plan, const cs_layer *layer, const float *x_host, int32_t B,
@@ -202,8 +247,11 @@ cs_status cs_ffn_exec_shared(cs_plan *plan, const cs_layer *layer, const void *H
     cs_status s = check_weights(layer);
     if (s != CS_OK) return s;
     if (n <= 0 || n > plan->cfg.max_tokens) return CS_ERR_SHAPE;
-    (void)stream;
-    return CS_ERR_UNSUPPORTED;
+    if (!plan->mma_ok || !aligned16(H) || !aligned16(out)) return CS_ERR_UNSUPPORTED;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    s = launch_check_support(plan, support, 1, st);
+    if (s != CS_OK) return s;
+    return launch_ffn_mma(plan, layer, H, nullptr, n, support, nullptr, plan->cfg.k, nullptr, nullptr, nullptr, out, st);
 }
 
 cs_status cs_last_device_status(cs_plan *plan, void *stream, int32_t *code) {

@@ -16,6 +16,7 @@ constexpr int kGatherThreads = 512;
 constexpr int kGatherMaxRows = 32;   // channel rows one gather CTA owns at most
 constexpr int kGatherMaxTokens = 16; // tokens per gather launch (scratch for partial sums)
 constexpr int kReduceGroups = 32;    // partial-sum groups of the deterministic cross-CTA reduction
+constexpr int kMmaMinTokens = 16;    // decode batches at least this large run on the tensor cores
 
 // Device status word values mirror cs_status (0 = ok).
 struct DeviceStatus {
@@ -39,6 +40,19 @@ struct cs_plan {
     float *hbar;       // [d] mean prompt hidden state
     float *colsum;     // [mean_row_blocks, d]
     cs::DeviceStatus *status;  // device status word
+    // tensor-core path (bf16 weights, 128-channel groups, d a multiple of 256)
+    uint32_t *mask;      // [max_tokens, 4] membership bits: bit g of token t
+    int32_t *counts;     // [G] tokens per group
+    int32_t *offsets;    // [G + 1]
+    int32_t *token_ids;  // [max_tokens * k] tokens of each group, ascending
+    int32_t *glist;      // [G] groups with a non-empty bucket, ascending
+    int32_t *nu;         // [1] their number
+    void *x_bf16;        // [2][max_tokens, d] bf16 activations: rounded value, then remainder
+    void *act;           // [2][max_tokens, d_ff] bf16 SwiGLU activations over the group list (value, remainder)
+    float *mma_partial;  // [slices, padded tokens, d] f32 partial down projections
+    int mma_ok;          // shape qualifies for the tensor-core path
+    int mma_slices;      // most list slices the down GEMM is split into
+    int last_slices;
     float *x_host_in;  // [max_tokens, d] staging for the host-buffer entry point
     float *x_host_out; // [max_tokens, d]
     cudaEvent_t ev[2 * CS_STAGE_COUNT];  // start/stop per stage
@@ -80,6 +94,13 @@ cs_status launch_ffn_gather(cs_plan *plan, const cs_layer *layer, const float *h
                             int B, const float *residual, float *out, cudaStream_t st);
 cs_status prepare_ffn_gather(cs_plan *plan);
 cs_status launch_check_support(cs_plan *plan, const int32_t *support, int B, cudaStream_t st);
+cs_status prepare_ffn_mma(cs_plan *plan);
+cs_status launch_bucket(cs_plan *plan, const int32_t *support, int B, cudaStream_t st, int32_t *counts = nullptr,
+                        int32_t *offsets = nullptr, int32_t *token_ids = nullptr);
+cs_status launch_split_bf16(cs_plan *plan, const float *x, void *y_hi, void *y_lo, size_t n, cudaStream_t st);
+cs_status launch_ffn_mma(cs_plan *plan, const cs_layer *L, const void *X, const void *X_lo, int M, const int32_t *glist,
+                         const int32_t *ng_dev, int ng_host, const uint32_t *mask, const float *residual,
+                         float *out_f32, void *out_bf16, cudaStream_t st);
 cs_status launch_prompt_mean(cs_plan *plan, const void *H, int n, float *hbar, cudaStream_t st);
 
 // ---- small device helpers -------------------------------------------------------------------

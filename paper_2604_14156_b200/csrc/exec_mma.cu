@@ -1,0 +1,545 @@
+// Actuator, tensor-core regime: the FFN over a list of active groups as two grouped GEMMs on the
+// 5th-generation tensor cores (tcgen05.mma, accumulators in tensor memory, operands fed by TMA).
+//
+//   gate/up  (ffn_gateup_mma_kernel):  for group g of the list and a tile of 128 tokens
+//        D[128 tokens, 256] = X[128, d] * [W_gate[g rows]; W_up[g rows]]^T      (bf16 x bf16 -> f32)
+//        act[token, slot*128 + c] = silu(D[:, c]) * D[:, 128 + c]  (* membership mask), as bf16
+//   down     (ffn_down_mma_kernel):    for a tile of 128 tokens, 256 output columns, a slice of the list
+//        P[128, 256] = act[128, slice] * Wd_t[slice rows, 256 columns]
+//   then out = residual + sum over slices of P (reduce_slices_kernel).
+//
+// The same kernels serve both uses of the paper's method: the prompt-level variant (one support
+// shared by every token: list = that support, no mask) and large decode batches with independent
+// supports (list = union of the supports, mask = which token owns which group).  With at most 128
+// tokens a single 128-row MMA tile holds every token, so "bucketing tokens by group" costs nothing
+// extra: the bucket of a group is the set of rows whose mask bit is set, and rows outside the bucket
+// are zeroed in the epilogue.  (Smaller MMA tiles would not be cheaper: the instruction's cost is
+// set by the 128-row weight operand it reads from shared memory.)
+//
+// Operand layouts (all 128-byte swizzled, written by TMA, read through shared-memory descriptors):
+//   X, act, W_gate, W_up tiles are K-major: [rows][64 k] with 128-byte rows, 8-row swizzle atoms.
+//   Wd_t tiles are N-major (the 256 output columns are contiguous in memory): four blocks of
+//   [64 k rows][64 columns], 8 KB each.
+//
+// One CTA per tile, six warps: warp 0 issues TMA, warp 1 owns tensor memory and issues the MMAs
+// (one elected lane), warps 2-5 run the epilogue (one warp per 32 TMEM lanes).  Every wait on an
+// mbarrier is bounded; a wait that runs out records CS_ERR_TIMEOUT in the plan's status word and the
+// CTA drains and exits.
+#include <cuda.h>
+
+#include "cs_internal.cuh"
+
+namespace cs {
+
+namespace {
+
+constexpr int BM = 128, BN = 256, BK = 64;
+constexpr int kMaxStages = 4;
+constexpr int kABytes = BM * BK * 2;   // 16 KB
+constexpr int kBBytes = BN * BK * 2;   // 32 KB
+constexpr int kRingBytesMma = 4 * (kABytes + kBBytes);   // 192 KB of operand tiles
+constexpr int kMmaThreads = 192;
+constexpr uint32_t kSpinLimit = 1u << 20;
+constexpr size_t kMmaSmem = 1024 + (size_t)kRingBytesMma + 256;
+
+struct Barriers {
+    uint64_t full[kMaxStages];
+    uint64_t empty[kMaxStages];
+    uint64_t acc_ready;
+    uint32_t tmem_base;
+    uint32_t aborted;
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) {
+    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+// Bounded wait on a phase parity.  Returns false (after flagging the timeout) if the limit is hit.
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, Barriers *bars, DeviceStatus *status) {
+    const uint32_t addr = smem_u32(bar);
+    for (uint32_t spin = 0; spin < kSpinLimit; ++spin) {
+        uint32_t done;
+        asm volatile(
+            "{\n.reg .pred p;\n"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+            "selp.u32 %0, 1, 0, p;\n}"
+            : "=r"(done) : "r"(addr), "r"(parity) : "memory");
+        if (done) return true;
+        if (*reinterpret_cast<volatile uint32_t *>(&bars->aborted)) return false;
+    }
+    bars->aborted = 1;
+    atomicCAS(&status->code, 0, (int)CS_ERR_TIMEOUT);
+    return false;
+}
+__device__ __forceinline__ void tma_load_2d(void *dst, const CUtensorMap *map, int x, int y, uint64_t *bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(smem_u32(dst)), "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint64_t *bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void tc_mma(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
+        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// 32 consecutive f32 columns of this warp's 32 TMEM lanes.
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptors (version 1, 128-byte swizzle).  Offsets are in 16-byte units.
+//   K-major:  rows 128 bytes apart, 8-row atoms 1024 bytes apart (SBO); LBO unused.
+//   MN-major: 64-element blocks `lbo_bytes` apart (LBO), 8-row k groups 1024 bytes apart (SBO).
+__device__ __forceinline__ uint64_t desc_sw128(uint32_t saddr, uint32_t lbo_bytes) {
+    uint64_t d = 0;
+    d |= (uint64_t)((saddr & 0x3ffff) >> 4);
+    d |= (uint64_t)(lbo_bytes >> 4) << 16;
+    d |= (uint64_t)(1024 >> 4) << 32;
+    d |= (uint64_t)1 << 46;   // descriptor version
+    d |= (uint64_t)2 << 61;   // SWIZZLE_128B
+    return d;
+}
+// Instruction descriptor: bf16 x bf16 -> f32, M = 128, N = 256; b_mn = B operand is N-major.
+__host__ __device__ constexpr uint32_t make_idesc(bool b_mn) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn ? 1u : 0u) << 16) | ((uint32_t)(BN >> 3) << 17) |
+           ((uint32_t)(BM >> 4) << 24);
+}
+
+// SPLIT: the activation operand comes as two bf16 matrices (high part and remainder, whose sum
+// carries ~16 mantissa bits), each stage holds both A tiles and every MMA is issued twice.  The
+// ring then has three stages of 64 KB instead of four of 48 KB.
+template <bool SPLIT> struct Ring {
+    static constexpr int kStages = SPLIT ? 3 : 4;
+    static constexpr int kStageBytes = (SPLIT ? 2 : 1) * kABytes + kBBytes;
+    static constexpr int kTxBytes = kStageBytes;
+};
+template <bool SPLIT> struct Tiles {
+    uint8_t *base;    // 1024-byte aligned; stage s holds its A tile(s) then its B tile
+    Barriers *bars;
+    __device__ __forceinline__ uint8_t *a(int s) const { return base + (size_t)s * Ring<SPLIT>::kStageBytes; }
+    __device__ __forceinline__ uint8_t *a_lo(int s) const { return a(s) + kABytes; }
+    __device__ __forceinline__ uint8_t *b(int s) const { return a(s) + (SPLIT ? 2 : 1) * kABytes; }
+};
+template <bool SPLIT> __device__ __forceinline__ Tiles<SPLIT> carve(uint8_t *raw) {
+    Tiles<SPLIT> t;
+    t.base = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(raw) + 1023) & ~(uintptr_t)1023);
+    t.bars = reinterpret_cast<Barriers *>(t.base + (size_t)kRingBytesMma);
+    return t;
+}
+
+// Common prologue: barriers, tensor memory (256 columns, owned by warp 1).
+template <bool SPLIT> __device__ __forceinline__ void prologue(const Tiles<SPLIT> &t, int warp, int lane) {
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kMaxStages; ++s) { mbar_init(&t.bars->full[s], 1); mbar_init(&t.bars->empty[s], 1); }
+        mbar_init(&t.bars->acc_ready, 1);
+        t.bars->aborted = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(&t.bars->tmem_base)), "r"(256) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    (void)lane;
+}
+template <bool SPLIT> __device__ __forceinline__ void epilogue_done(const Tiles<SPLIT> &t, int warp) {
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(t.bars->tmem_base), "r"(256) : "memory");
+    }
+}
+
+// The MMA issue loop shared by both kernels: `kblocks` stages of four K=16 instructions.
+template <bool B_MN, bool SPLIT>
+__device__ __forceinline__ void mma_loop(const Tiles<SPLIT> &t, int kblocks, DeviceStatus *status) {
+    constexpr uint32_t idesc = make_idesc(B_MN);
+    constexpr int kStages = Ring<SPLIT>::kStages;
+    const uint32_t tmem = t.bars->tmem_base;
+    for (int kb = 0; kb < kblocks; ++kb) {
+        const int s = kb % kStages;
+        if (!mbar_wait(&t.bars->full[s], (kb / kStages) & 1, t.bars, status)) return;
+        tc_fence_after();
+        const uint32_t a0 = smem_u32(t.a(s)), a1 = smem_u32(t.a_lo(s)), b0 = smem_u32(t.b(s));
+#pragma unroll
+        for (int k4 = 0; k4 < BK / 16; ++k4) {
+            const uint64_t bd = B_MN ? desc_sw128(b0 + k4 * 2048, 64 * BK * 2) : desc_sw128(b0 + k4 * 32, 16);
+            tc_mma(tmem, desc_sw128(a0 + k4 * 32, 16), bd, idesc, (kb | k4) != 0);
+            if (SPLIT) tc_mma(tmem, desc_sw128(a1 + k4 * 32, 16), bd, idesc, 1);
+        }
+        tc_commit(&t.bars->empty[s]);   // frees the stage once these MMAs have read it
+    }
+    tc_commit(&t.bars->acc_ready);
+}
+
+__device__ __forceinline__ float silu_f(float x) { return x / (1.f + __expf(-x)); }
+
+}  // namespace
+
+// ---- gate / up --------------------------------------------------------------------------------
+template <bool SPLIT>
+__global__ void __launch_bounds__(kMmaThreads, 1)
+ffn_gateup_mma_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_x_lo,
+                      const __grid_constant__ CUtensorMap tm_g, const __grid_constant__ CUtensorMap tm_u,
+                      const int32_t *__restrict__ glist, const int32_t *__restrict__ ng_dev, int ng_host, int M,
+                      int d, int act_ld, const uint32_t *__restrict__ mask, __nv_bfloat16 *__restrict__ act,
+                      __nv_bfloat16 *__restrict__ act_lo, DeviceStatus *status) {
+    constexpr int kStages = Ring<SPLIT>::kStages;
+    extern __shared__ uint8_t smem_raw[];
+    const int gi = blockIdx.x, mt = blockIdx.y;
+    const int ng = ng_dev != nullptr ? *ng_dev : ng_host;
+    if (gi >= ng) return;
+    const int g = glist[gi];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const Tiles<SPLIT> t = carve<SPLIT>(smem_raw);
+    prologue(t, warp, lane);
+    const int kblocks = d / BK;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            for (int kb = 0; kb < kblocks; ++kb) {
+                const int s = kb % kStages;
+                if (kb >= kStages && !mbar_wait(&t.bars->empty[s], ((kb / kStages) - 1) & 1, t.bars, status)) break;
+                mbar_expect_tx(&t.bars->full[s], Ring<SPLIT>::kTxBytes);
+                tma_load_2d(t.a(s), &tm_x, kb * BK, mt * BM, &t.bars->full[s]);
+                if (SPLIT) tma_load_2d(t.a_lo(s), &tm_x_lo, kb * BK, mt * BM, &t.bars->full[s]);
+                tma_load_2d(t.b(s), &tm_g, kb * BK, g * 128, &t.bars->full[s]);
+                tma_load_2d(t.b(s) + kBBytes / 2, &tm_u, kb * BK, g * 128, &t.bars->full[s]);
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) mma_loop<false, SPLIT>(t, kblocks, status);
+    } else {
+        const int q = warp & 3;                    // TMEM lane quarter this warp may read
+        const int row = q * 32 + lane, m = mt * BM + row;
+        if (mbar_wait(&t.bars->acc_ready, 0, t.bars, status)) {
+            tc_fence_after();
+            const uint32_t tbase = t.bars->tmem_base + ((uint32_t)(q * 32) << 16);
+            float keep = 1.f;
+            if (mask != nullptr && m < M) keep = ((mask[(size_t)m * 4 + (g >> 5)] >> (g & 31)) & 1u) ? 1.f : 0.f;
+#pragma unroll 1
+            for (int c = 0; c < 4; ++c) {
+                uint32_t gv[32], uv[32];
+                tc_ld32(tbase + c * 32, gv);
+                tc_ld32(tbase + 128 + c * 32, uv);
+                tc_wait_ld();
+                uint32_t packed[16], packed_lo[16];
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                    const float a0 = silu_f(__uint_as_float(gv[2 * j])) * __uint_as_float(uv[2 * j]) * keep;
+                    const float a1 = silu_f(__uint_as_float(gv[2 * j + 1])) * __uint_as_float(uv[2 * j + 1]) * keep;
+                    const __nv_bfloat162 p = __floats2bfloat162_rn(a0, a1);
+                    packed[j] = *reinterpret_cast<const uint32_t *>(&p);
+                    if (SPLIT) {
+                        const __nv_bfloat162 r = __floats2bfloat162_rn(a0 - __low2float(p), a1 - __high2float(p));
+                        packed_lo[j] = *reinterpret_cast<const uint32_t *>(&r);
+                    }
+                }
+                if (m < M) {
+                    const size_t off = (size_t)m * act_ld + (size_t)gi * 128 + c * 32;
+                    uint4 *dst = reinterpret_cast<uint4 *>(act + off);
+#pragma unroll
+                    for (int j = 0; j < 4; ++j)
+                        dst[j] = make_uint4(packed[4 * j], packed[4 * j + 1], packed[4 * j + 2], packed[4 * j + 3]);
+                    if (SPLIT) {
+                        uint4 *dlo = reinterpret_cast<uint4 *>(act_lo + off);
+#pragma unroll
+                        for (int j = 0; j < 4; ++j)
+                            dlo[j] = make_uint4(packed_lo[4 * j], packed_lo[4 * j + 1], packed_lo[4 * j + 2], packed_lo[4 * j + 3]);
+                    }
+                }
+            }
+        }
+    }
+    epilogue_done(t, warp);
+}
+
+// ---- down -------------------------------------------------------------------------------------
+// grid (d / 256, token tiles, slices).  Slice z covers list entries [z*ng/Z, (z+1)*ng/Z).
+template <bool SPLIT>
+__global__ void __launch_bounds__(kMmaThreads, 1)
+ffn_down_mma_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant__ CUtensorMap tm_act_lo,
+                    const __grid_constant__ CUtensorMap tm_wd, const int32_t *__restrict__ glist,
+                    const int32_t *__restrict__ ng_dev, int ng_host, int M, int m_pad, int d,
+                    float *__restrict__ partial, DeviceStatus *status) {
+    constexpr int kStages = Ring<SPLIT>::kStages;
+    extern __shared__ uint8_t smem_raw[];
+    const int nt = blockIdx.x, mt = blockIdx.y, z = blockIdx.z, Z = gridDim.z;
+    const int ng = ng_dev != nullptr ? *ng_dev : ng_host;
+    const int gi0 = (int)(((long long)ng * z) / Z), gi1 = (int)(((long long)ng * (z + 1)) / Z);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const Tiles<SPLIT> t = carve<SPLIT>(smem_raw);
+    prologue(t, warp, lane);
+    const int kblocks = (gi1 - gi0) * 2;   // two 64-row k blocks per 128-channel group
+
+    if (warp == 0) {
+        if (lane == 0) {
+            for (int kb = 0; kb < kblocks; ++kb) {
+                const int s = kb % kStages;
+                if (kb >= kStages && !mbar_wait(&t.bars->empty[s], ((kb / kStages) - 1) & 1, t.bars, status)) break;
+                const int gi = gi0 + (kb >> 1), half = kb & 1;
+                const int wrow = glist[gi] * 128 + half * BK;
+                mbar_expect_tx(&t.bars->full[s], Ring<SPLIT>::kTxBytes);
+                tma_load_2d(t.a(s), &tm_act, gi * 128 + half * BK, mt * BM, &t.bars->full[s]);
+                if (SPLIT) tma_load_2d(t.a_lo(s), &tm_act_lo, gi * 128 + half * BK, mt * BM, &t.bars->full[s]);
+#pragma unroll
+                for (int j = 0; j < BN / 64; ++j)
+                    tma_load_2d(t.b(s) + j * (64 * BK * 2), &tm_wd, nt * BN + j * 64, wrow, &t.bars->full[s]);
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0 && kblocks > 0) mma_loop<true, SPLIT>(t, kblocks, status);
+    } else {
+        const int q = warp & 3;
+        const int row = q * 32 + lane, m = mt * BM + row;
+        float *dst = partial + ((size_t)z * m_pad + m) * d + (size_t)nt * BN;
+        if (kblocks == 0) {   // empty slice: its partial is zero
+            if (m < M) for (int c = 0; c < BN; c += 4) *reinterpret_cast<float4 *>(dst + c) = make_float4(0.f, 0.f, 0.f, 0.f);
+        } else if (mbar_wait(&t.bars->acc_ready, 0, t.bars, status)) {
+            tc_fence_after();
+            const uint32_t tbase = t.bars->tmem_base + ((uint32_t)(q * 32) << 16);
+#pragma unroll 1
+            for (int c = 0; c < BN / 32; ++c) {
+                uint32_t v[32];
+                tc_ld32(tbase + c * 32, v);
+                tc_wait_ld();
+                if (m < M) {
+#pragma unroll
+                    for (int j = 0; j < 8; ++j)
+                        *reinterpret_cast<uint4 *>(dst + c * 32 + 4 * j) = make_uint4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+                }
+            }
+        }
+    }
+    epilogue_done(t, warp);
+}
+
+// out[m, :] = residual[m, :] + sum_z partial[z, m, :], slices added in index order.
+template <typename OutT>
+__global__ void reduce_slices_kernel(const float *__restrict__ partial, int Z, int M, int m_pad, int d,
+                                     const float *__restrict__ residual, OutT *__restrict__ out) {
+    const size_t i4 = (size_t)blockIdx.x * blockDim.x + threadIdx.x;   // float4 index
+    const size_t total4 = (size_t)M * d / 4;
+    if (i4 >= total4) return;
+    const size_t m = (i4 * 4) / d, c = (i4 * 4) % d;
+    float4 s = residual != nullptr ? *reinterpret_cast<const float4 *>(residual + m * d + c) : make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int z = 0; z < Z; ++z) {
+        const float4 v = *reinterpret_cast<const float4 *>(partial + ((size_t)z * m_pad + m) * d + c);
+        s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
+    }
+    if constexpr (sizeof(OutT) == 4) {
+        *reinterpret_cast<float4 *>(reinterpret_cast<float *>(out) + m * d + c) = s;
+    } else {
+        const __nv_bfloat162 lo = __floats2bfloat162_rn(s.x, s.y), hi = __floats2bfloat162_rn(s.z, s.w);
+        uint2 p;
+        p.x = *reinterpret_cast<const uint32_t *>(&lo);
+        p.y = *reinterpret_cast<const uint32_t *>(&hi);
+        *reinterpret_cast<uint2 *>(reinterpret_cast<__nv_bfloat16 *>(out) + m * d + c) = p;
+    }
+}
+
+// x = y_hi + y_lo with both parts bf16: y_hi = round(x), y_lo = round(x - y_hi).
+__global__ void split_bf16_kernel(const float *__restrict__ x, __nv_bfloat16 *__restrict__ y_hi,
+                                  __nv_bfloat16 *__restrict__ y_lo, size_t n4) {
+    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n4) return;
+    const float4 v = reinterpret_cast<const float4 *>(x)[i];
+    const __nv_bfloat162 h0 = __floats2bfloat162_rn(v.x, v.y), h1 = __floats2bfloat162_rn(v.z, v.w);
+    const __nv_bfloat162 l0 = __floats2bfloat162_rn(v.x - __low2float(h0), v.y - __high2float(h0));
+    const __nv_bfloat162 l1 = __floats2bfloat162_rn(v.z - __low2float(h1), v.w - __high2float(h1));
+    uint2 p, q;
+    p.x = *reinterpret_cast<const uint32_t *>(&h0); p.y = *reinterpret_cast<const uint32_t *>(&h1);
+    q.x = *reinterpret_cast<const uint32_t *>(&l0); q.y = *reinterpret_cast<const uint32_t *>(&l1);
+    reinterpret_cast<uint2 *>(y_hi)[i] = p;
+    reinterpret_cast<uint2 *>(y_lo)[i] = q;
+}
+
+// ---- bucketing: supports [B,k] -> membership masks, per-group token lists, union list ------------
+// One CTA.  mask [B][4] (bit g of token t), counts [G], offsets [G+1], token_ids [B*k] (tokens of
+// group g ascending at offsets[g]..offsets[g+1]), glist [G] (groups with a non-empty bucket,
+// ascending), *nu = their number.
+__global__ void __launch_bounds__(1024)
+bucket_kernel(const int32_t *__restrict__ support, int B, int k, int G, uint32_t *__restrict__ mask,
+              int32_t *__restrict__ counts, int32_t *__restrict__ offsets, int32_t *__restrict__ token_ids,
+              int32_t *__restrict__ glist, int32_t *__restrict__ nu) {
+    __shared__ int cnt_s[kMaxG];
+    __shared__ int off_s[kMaxG + 1];
+    const int tid = threadIdx.x;
+    if (tid < kMaxG) cnt_s[tid] = 0;
+    __syncthreads();
+    for (int t = tid; t < B; t += blockDim.x) {
+        uint32_t w[4] = {0u, 0u, 0u, 0u};
+        for (int c = 0; c < k; ++c) {
+            const int g = support[(size_t)t * k + c];
+            if (g >= 0 && g < G) { w[g >> 5] |= 1u << (g & 31); atomicAdd(&cnt_s[g], 1); }
+        }
+        *reinterpret_cast<uint4 *>(mask + (size_t)t * 4) = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+    __syncthreads();
+    if (tid == 0) {
+        int run = 0, n = 0;
+        for (int g = 0; g < G; ++g) {
+            off_s[g] = run; run += cnt_s[g];
+            if (cnt_s[g] > 0) glist[n++] = g;
+        }
+        off_s[G] = run;
+        *nu = n;
+    }
+    __syncthreads();
+    if (tid < G) { counts[tid] = cnt_s[tid]; offsets[tid] = off_s[tid]; }
+    if (tid == 0) offsets[G] = off_s[G];
+    // token lists in ascending token order: thread g walks the tokens (the masks were just written
+    // by this CTA; make them visible first)
+    __threadfence_block();
+    __syncthreads();
+    if (tid < G) {
+        int o = off_s[tid];
+        for (int t = 0; t < B; ++t)
+            if ((mask[(size_t)t * 4 + (tid >> 5)] >> (tid & 31)) & 1u) token_ids[o++] = t;
+    }
+}
+
+// ---- host side ----------------------------------------------------------------------------------
+namespace {
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (fn == nullptr) {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// bf16 matrix [outer, inner] row-major with `ld` elements per row; box = [box_outer rows, 64 columns].
+bool make_map(CUtensorMap *map, const void *base, uint64_t inner, uint64_t outer, uint64_t ld, uint32_t box_outer) {
+    EncodeTiledFn fn = encode_fn();
+    if (fn == nullptr) return false;
+    const cuuint64_t dims[2] = {inner, outer};
+    const cuuint64_t strides[1] = {ld * 2};
+    const cuuint32_t box[2] = {64, box_outer};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+cs_status prepare_ffn_mma(cs_plan *plan) {
+    CS_CUDA_TRY(plan, cudaFuncSetAttribute(ffn_gateup_mma_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMmaSmem));
+    CS_CUDA_TRY(plan, cudaFuncSetAttribute(ffn_gateup_mma_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMmaSmem));
+    CS_CUDA_TRY(plan, cudaFuncSetAttribute(ffn_down_mma_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMmaSmem));
+    CS_CUDA_TRY(plan, cudaFuncSetAttribute(ffn_down_mma_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMmaSmem));
+    return CS_OK;
+}
+
+cs_status launch_bucket(cs_plan *plan, const int32_t *support, int B, cudaStream_t st, int32_t *counts,
+                        int32_t *offsets, int32_t *token_ids) {
+    bucket_kernel<<<1, 1024, 0, st>>>(support, B, plan->cfg.k, plan->G, plan->mask,
+                                      counts ? counts : plan->counts, offsets ? offsets : plan->offsets,
+                                      token_ids ? token_ids : plan->token_ids, plan->glist, plan->nu);
+    plan->launches++;
+    CS_CUDA_TRY(plan, cudaGetLastError());
+    return CS_OK;
+}
+
+// X [M, d] bf16 (plus X_lo, the bf16 remainder, when split precision is wanted); list / count on the
+// device (ng_dev) or count on the host; mask may be NULL.  Writes out [M, d] as f32 (out_f32) or bf16
+// (out_bf16), plus residual (f32, may be NULL).
+cs_status launch_ffn_mma(cs_plan *plan, const cs_layer *L, const void *X, const void *X_lo, int M,
+                         const int32_t *glist, const int32_t *ng_dev, int ng_host, const uint32_t *mask,
+                         const float *residual, float *out_f32, void *out_bf16, cudaStream_t st) {
+    const cs_config &c = plan->cfg;
+    const bool split = X_lo != nullptr;
+    const int grid_g = ng_dev != nullptr ? plan->G : ng_host;       // CTAs past the device count exit at once
+    const int act_ld = plan->G * 128;
+    const int mtiles = (M + BM - 1) / BM, m_pad = mtiles * BM;
+    __nv_bfloat16 *act = static_cast<__nv_bfloat16 *>(plan->act);
+    __nv_bfloat16 *act_lo = act + (size_t)plan->cfg.max_tokens * act_ld;
+    CUtensorMap tm_x, tm_x_lo, tm_g, tm_u, tm_act, tm_act_lo, tm_wd;
+    if (!make_map(&tm_x, X, c.d, M, c.d, BM) || !make_map(&tm_x_lo, split ? X_lo : X, c.d, M, c.d, BM) ||
+        !make_map(&tm_g, L->W_gate, c.d, c.d_ff, c.d, 128) || !make_map(&tm_u, L->W_up, c.d, c.d_ff, c.d, 128) ||
+        !make_map(&tm_act, act, act_ld, M, act_ld, BM) ||
+        !make_map(&tm_act_lo, split ? act_lo : act, act_ld, M, act_ld, BM) ||
+        !make_map(&tm_wd, L->Wd_t, c.d, c.d_ff, c.d, BK))
+        return record_cuda(plan, cudaErrorInvalidValue, "cuTensorMapEncodeTiled");
+    {
+        StageTimer timer(plan, CS_STAGE_EXEC, st);
+        if (split)
+            ffn_gateup_mma_kernel<true><<<dim3(grid_g, mtiles), kMmaThreads, kMmaSmem, st>>>(
+                tm_x, tm_x_lo, tm_g, tm_u, glist, ng_dev, ng_host, M, c.d, act_ld, mask, act, act_lo, plan->status);
+        else
+            ffn_gateup_mma_kernel<false><<<dim3(grid_g, mtiles), kMmaThreads, kMmaSmem, st>>>(
+                tm_x, tm_x_lo, tm_g, tm_u, glist, ng_dev, ng_host, M, c.d, act_ld, mask, act, act_lo, plan->status);
+        plan->launches++;
+        CS_CUDA_TRY(plan, cudaGetLastError());
+        // slices: fill the machine when one token tile cannot (decode), one slice otherwise (prompt)
+        const int ntiles = c.d / BN;
+        int Z = 1;
+        if (mtiles * ntiles < plan->sm_count) Z = max(1, min(plan->sm_count / (mtiles * ntiles), plan->mma_slices));
+        if (split)
+            ffn_down_mma_kernel<true><<<dim3(ntiles, mtiles, Z), kMmaThreads, kMmaSmem, st>>>(
+                tm_act, tm_act_lo, tm_wd, glist, ng_dev, ng_host, M, m_pad, c.d, plan->mma_partial, plan->status);
+        else
+            ffn_down_mma_kernel<false><<<dim3(ntiles, mtiles, Z), kMmaThreads, kMmaSmem, st>>>(
+                tm_act, tm_act_lo, tm_wd, glist, ng_dev, ng_host, M, m_pad, c.d, plan->mma_partial, plan->status);
+        plan->launches++;
+        CS_CUDA_TRY(plan, cudaGetLastError());
+        plan->last_slices = Z;
+    }
+    {
+        StageTimer timer(plan, CS_STAGE_REDUCE, st);
+        const size_t total4 = (size_t)M * c.d / 4;
+        const int blocks = (int)((total4 + 255) / 256);
+        if (out_f32 != nullptr)
+            reduce_slices_kernel<float><<<blocks, 256, 0, st>>>(plan->mma_partial, plan->last_slices, M, m_pad, c.d, residual, out_f32);
+        else
+            reduce_slices_kernel<__nv_bfloat16><<<blocks, 256, 0, st>>>(plan->mma_partial, plan->last_slices, M, m_pad, c.d,
+                                                                       residual, static_cast<__nv_bfloat16 *>(out_bf16));
+        plan->launches++;
+        CS_CUDA_TRY(plan, cudaGetLastError());
+    }
+    return CS_OK;
+}
+
+cs_status launch_split_bf16(cs_plan *plan, const float *x, void *y_hi, void *y_lo, size_t n, cudaStream_t st) {
+    const size_t n4 = n / 4;
+    split_bf16_kernel<<<(unsigned)((n4 + 255) / 256), 256, 0, st>>>(x, static_cast<__nv_bfloat16 *>(y_hi),
+                                                                   static_cast<__nv_bfloat16 *>(y_lo), n4);
+    plan->launches++;
+    CS_CUDA_TRY(plan, cudaGetLastError());
+    return CS_OK;
+}
+
+}  // namespace cs
