@@ -40,18 +40,21 @@ def parse_args():
     ap.add_argument("--steps", type=int, default=20000)
     ap.add_argument("--warmup", type=int, default=200)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
-    ap.add_argument("--workload", default="l2_7b_b1", choices=["l2_7b_b1", "l2_7b_b64", "l3_8b_stack", "tiny_f32"])
+    ap.add_argument("--workload", default="l2_7b_b1",
+                    choices=["l2_7b_b1", "l2_7b_b64", "l3_8b_stack", "tiny_f32", "l2_13b_prompt"])
+    ap.add_argument("--k", type=int, default=0, help="active groups (prompt workload sweep: 11 / 27 / 54)")
     ap.add_argument("--layers", type=int, default=0, help="distinct layers rotated through (0 = auto)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     return ap.parse_args()
 
 
 def peaks():
+    """(HBM GB/s, sustained bf16 TFLOP/s, 'measured' | 'fallback')."""
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
         p = json.load(open(path))
-        return float(p["hbm_gbs"]), "measured"
-    return 6650.0, "fallback"
+        return float(p["hbm_gbs"]), float(p.get("bf16_tflops_sustained", p.get("bf16_tflops", 1400.0))), "measured"
+    return 6650.0, 1400.0, "fallback"
 
 
 class ClockSampler:
@@ -132,6 +135,10 @@ def run_ours(args):
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=dev)
     cfg = W.CONFIGS[args.workload]
+    if args.k:
+        cfg = cfg.with_(k=args.k)
+    if cfg.prompt:
+        return run_prompt(args, cfg, rank, world, local, dev)
     wbytes_layer = 3 * cfg.d_ff * cfg.d * (2 if cfg.w_dtype == "bf16" else 4)
     n_layers = args.layers or (cfg.n_layers if cfg.n_layers > 1 else max(8, int(4e9 // wbytes_layer)))
     n_layers = min(n_layers, GRAPH_STEPS)
@@ -150,8 +157,14 @@ def run_ours(args):
     x_out = torch.empty_like(xs[0])
     sup_probe = None
 
+    chained = cfg.n_layers > 1   # the stack: each layer's input is the previous layer's output
+    x_chain = xs[0].clone()
+
     def step(i):
-        cs.cs_layer_step(plan, layers[i % n_layers], xs[i % N_TOKEN_BATCHES], x_out=x_out, want_aux=False)
+        if chained:
+            cs.cs_layer_step(plan, layers[i % n_layers], x_chain, x_out=x_chain, want_aux=False)
+        else:
+            cs.cs_layer_step(plan, layers[i % n_layers], xs[i % N_TOKEN_BATCHES], x_out=x_out, want_aux=False)
 
     stream = torch.cuda.Stream(device=dev)
     chunk = min(K, GRAPH_STEPS)
@@ -239,8 +252,9 @@ def run_ours(args):
     tokens = cfg.B * K * world
     value = tokens / (ms_total * 1e-3)
     ab = algorithmic_bytes(cfg, union)
-    peak, peak_kind = peaks()
+    peak, _, peak_kind = peaks()
     exec_ms = stage_ms[2]
+    mma = cfg.B >= 16 and cfg.w_dtype == "bf16" and cfg.group == 128
     # the dominant kernel reads the active weights and the hidden state, writes its partial sums
     kernel_bytes = ab["weights"] + cfg.B * cfg.d * 4 * 2
     achieved = kernel_bytes / (exec_ms * 1e-3) / 1e9 if exec_ms > 0 else None
@@ -259,7 +273,9 @@ def run_ours(args):
                 "d2h_bytes_per_step": cfg.B * cfg.d * 4},
         "gpu_launches": int(round(launches_per_step * K)),
         "clocks": clocks.summary(),
-        "roofline": {"bound": "hbm", "kernel": "ffn_gather_kernel", "achieved": achieved, "peak": peak,
+        "roofline": {"bound": "hbm",
+                     "kernel": "ffn_gateup_mma_kernel + ffn_down_mma_kernel" if mma else "ffn_gather_kernel",
+                     "achieved": achieved, "peak": peak,
                      "unit": "GB/s", "frac": (achieved / peak) if achieved else None, "peak_kind": peak_kind,
                      "frac_of_8tbs_nominal": (achieved / 8000.0) if achieved else None,
                      "bytes_per_launch": kernel_bytes, "avg_launch_us": exec_ms * 1e3, "traffic": None},
@@ -275,6 +291,103 @@ def run_ours(args):
         out["cpu_baseline"] = cpu_baseline(cfg, [L.to("cpu") for L in layers_raw[:2]], hx, seconds=12.0)
     if rank == 0:
         print(json.dumps(out))
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+def run_prompt(args, cfg, rank, world, local, dev):
+    """Prompt-level variant: one support from the mean prompt sketch, then the FFN of all 2048 prompt
+    tokens over that support as grouped GEMMs.  A step is one prompt through one layer."""
+    import paper_2604_14156_b200 as cs
+    K, Wm = args.steps, max(args.warmup, 3)
+    n_layers = args.layers or 8
+    plan = cs.Plan(cfg.d, cfg.d_ff, cfg.group, cfg.m, cfg.k, cfg.T, torch.bfloat16, cfg.B, cfg.rms_eps)
+    raw = [W.make_layer(cfg, i, device=dev) for i in range(n_layers)]
+    layers = [cs.Layer(plan, L.S, L.Phi, L.W_gate, L.W_up, L.Wd_t, L.mu) for L in raw]
+    Hs = torch.stack([W.make_tokens(cfg, raw[0].A, batch=rank * 4 + j).h for j in range(4)]).to(dev)
+    out = torch.empty_like(Hs[0])
+
+    def step(i):
+        L = raw[i % n_layers]
+        s, _, _ = cs.cs_prompt_support(plan, L.S, L.Phi, L.mu, Hs[i % 4])
+        cs.cs_ffn_exec_shared(plan, layers[i % n_layers], Hs[i % 4], s, out=out)
+
+    def barrier():
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+
+    def timed(fn, n):
+        barrier(); torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(n):
+            fn(i)
+        e1.record()
+        torch.cuda.synchronize(); barrier()
+        ms = e0.elapsed_time(e1)
+        if world > 1:
+            import torch.distributed as dist
+            t = torch.tensor([ms], device=dev, dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms
+
+    for i in range(Wm):
+        step(i)
+    before = plan.launches
+    with ClockSampler(local) as clocks:
+        ms_total = timed(step, K)
+    launches = plan.launches - before
+    hH = Hs.cpu().pin_memory(); hout = torch.empty_like(hH[0]).pin_memory()
+    Hd = torch.empty_like(Hs[0])
+
+    def step_host(i):
+        Hd.copy_(hH[i % 4], non_blocking=True)
+        L = raw[i % n_layers]
+        s, _, _ = cs.cs_prompt_support(plan, L.S, L.Phi, L.mu, Hd)
+        cs.cs_ffn_exec_shared(plan, layers[i % n_layers], Hd, s, out=out)
+        hout.copy_(out, non_blocking=True)
+
+    for i in range(3):
+        step_host(i)
+    ms_e2e = timed(step_host, K)
+    plan.enable_timing(True)
+    acc = [0.0] * 4
+    n_prof = min(K, 50)
+    for i in range(n_prof + 3):
+        step(i)
+        t = plan.stage_times()
+        if i >= 3:
+            acc = [a + b for a, b in zip(acc, t)]
+    plan.enable_timing(False)
+    stage_ms = [a / n_prof for a in acc]
+    _, tf_peak, kind = peaks()
+    flops = 6.0 * cfg.B * cfg.k * cfg.group * cfg.d
+    achieved = flops / (stage_ms[2] * 1e-3) / 1e12
+    tokens = cfg.B * K * world
+    res = {
+        "metric": METRIC, "value": tokens / (ms_total * 1e-3), "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
+        "ms_per_step": ms_total / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": cfg.name, "d": cfg.d, "d_ff": cfg.d_ff, "groups": cfg.G, "group": cfg.group,
+                   "m": cfg.m, "k": cfg.k, "T": cfg.T, "prompt_tokens": cfg.B, "weights": "bf16",
+                   "accumulate": "f32", "layers_rotated": n_layers,
+                   "l2": f"inputs larger than L2: {n_layers} layers rotated, 4 prompts of {cfg.B * cfg.d * 2 / 1e6:.0f} MB",
+                   "e2e_path": "pinned host copies around the device entry points",
+                   "parallelism": f"dp{world}" if world > 1 else "single"},
+        "e2e": {"value": tokens / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": cfg.B * cfg.d * 2,
+                "d2h_bytes_per_step": cfg.B * cfg.d * 2},
+        "gpu_launches": launches, "clocks": clocks.summary(),
+        "roofline": {"bound": "tensor", "kernel": "ffn_gateup_mma_kernel + ffn_down_mma_kernel", "achieved": achieved,
+                     "peak": tf_peak, "unit": "TFLOP/s", "frac": achieved / tf_peak, "peak_kind": kind + " (sustained)",
+                     "flops_per_launch_pair": flops, "avg_pair_us": stage_ms[2] * 1e3, "traffic": None},
+        "stages_us": {"mean_sketch": stage_ms[0] * 1e3, "recover": stage_ms[1] * 1e3, "exec": stage_ms[2] * 1e3,
+                      "reduce": stage_ms[3] * 1e3, "step_net": ms_total * 1e3 / K},
+    }
+    if rank == 0:
+        print(json.dumps(res))
     if world > 1:
         import torch.distributed as dist
         dist.destroy_process_group()
