@@ -64,6 +64,7 @@ cs_status cs_plan_create(const cs_config *cfg, cs_plan **out) {
     alloc((void **)&p->status, sizeof(DeviceStatus));
     p->mma_ok = cfg->w_dtype == CS_BF16 && cfg->group == 128 && cfg->d % 256 == 0;
     alloc((void **)&p->mask, nt * 4 * sizeof(uint32_t));
+    alloc((void **)&p->gmask, (size_t)kMaxG * 4 * sizeof(uint32_t));
     alloc((void **)&p->counts, (size_t)kMaxG * sizeof(int32_t));
     alloc((void **)&p->offsets, (size_t)(kMaxG + 1) * sizeof(int32_t));
     alloc((void **)&p->token_ids, nt * cfg->k * sizeof(int32_t));
@@ -73,7 +74,7 @@ cs_status cs_plan_create(const cs_config *cfg, cs_plan **out) {
         const size_t m_pad = (nt + 127) / 128 * 128;
         p->mma_slices = max(1, min(16, p->sm_count / max(1, cfg->d / 256)));
         alloc((void **)&p->x_bf16, 2 * nt * cfg->d * 2);
-        alloc((void **)&p->act, 2 * nt * cfg->d_ff * 2);
+        alloc((void **)&p->act, 2 * max(nt, (size_t)128) * cfg->d_ff * 2);
         // slices * padded tokens never exceeds 128 * (SMs / column tiles): see launch_ffn_mma
         const size_t slice_rows = (size_t)128 * (p->sm_count / max(1, cfg->d / 256) + 1);
         alloc((void **)&p->mma_partial, max(slice_rows, m_pad) * cfg->d * sizeof(float));
@@ -98,7 +99,7 @@ cs_status cs_plan_destroy(cs_plan *p) {
     cudaFree(p->n_buf); cudaFree(p->y_buf); cudaFree(p->sup_buf); cudaFree(p->z_buf);
     cudaFree(p->resid_buf); cudaFree(p->partial); cudaFree(p->hbar); cudaFree(p->colsum);
     cudaFree(p->status); cudaFree(p->x_host_in); cudaFree(p->x_host_out);
-    cudaFree(p->mask); cudaFree(p->counts); cudaFree(p->offsets); cudaFree(p->token_ids); cudaFree(p->glist);
+    cudaFree(p->mask); cudaFree(p->gmask); cudaFree(p->counts); cudaFree(p->offsets); cudaFree(p->token_ids); cudaFree(p->glist);
     cudaFree(p->nu); cudaFree(p->x_bf16); cudaFree(p->act); cudaFree(p->mma_partial);
     for (int i = 0; i < 2 * CS_STAGE_COUNT; ++i)
         if (p->ev[i] != nullptr) cudaEventDestroy(p->ev[i]);
@@ -139,6 +140,7 @@ static cs_status exec_dispatch(cs_plan *plan, const cs_layer *layer, const float
     if (s != CS_OK) return s;
     s = launch_bucket(plan, support, B, st);
     if (s != CS_OK) return s;
+    if (B <= 128) return launch_ffn_mma_decode(plan, layer, x_hi, x_lo, B, residual, out, st);
     return launch_ffn_mma(plan, layer, x_hi, x_lo, B, plan->glist, plan->nu, 0, plan->mask, residual, out, nullptr, st);
 }
 

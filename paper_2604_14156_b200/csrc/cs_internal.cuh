@@ -42,6 +42,7 @@ struct cs_plan {
     cs::DeviceStatus *status;  // device status word
     // tensor-core path (bf16 weights, 128-channel groups, d a multiple of 256)
     uint32_t *mask;      // [max_tokens, 4] membership bits: bit g of token t
+    uint32_t *gmask;     // [G, 4] membership bits the other way round: bit t of group g (t < 128)
     int32_t *counts;     // [G] tokens per group
     int32_t *offsets;    // [G + 1]
     int32_t *token_ids;  // [max_tokens * k] tokens of each group, ascending
@@ -101,6 +102,8 @@ cs_status launch_split_bf16(cs_plan *plan, const float *x, void *y_hi, void *y_l
 cs_status launch_ffn_mma(cs_plan *plan, const cs_layer *L, const void *X, const void *X_lo, int M, const int32_t *glist,
                          const int32_t *ng_dev, int ng_host, const uint32_t *mask, const float *residual,
                          float *out_f32, void *out_bf16, cudaStream_t st);
+cs_status launch_ffn_mma_decode(cs_plan *plan, const cs_layer *L, const void *X, const void *X_lo, int B,
+                                const float *residual, float *out, cudaStream_t st);
 cs_status launch_prompt_mean(cs_plan *plan, const void *H, int n, float *hbar, cudaStream_t st);
 
 // ---- small device helpers -------------------------------------------------------------------

@@ -34,7 +34,7 @@ namespace cs {
 namespace {
 
 constexpr int BM = 128, BN = 256, BK = 64;
-constexpr int kMaxStages = 4;
+constexpr int kMaxStages = 8;
 constexpr int kABytes = BM * BK * 2;   // 16 KB
 constexpr int kBBytes = BN * BK * 2;   // 32 KB
 constexpr int kRingBytesMma = 4 * (kABytes + kBBytes);   // 192 KB of operand tiles
@@ -122,6 +122,46 @@ __device__ __forceinline__ uint64_t desc_sw128(uint32_t saddr, uint32_t lbo_byte
 __host__ __device__ constexpr uint32_t make_idesc(bool b_mn) {
     return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn ? 1u : 0u) << 16) | ((uint32_t)(BN >> 3) << 17) |
            ((uint32_t)(BM >> 4) << 24);
+}
+
+// General form: N columns, either operand MN-major.
+__device__ __forceinline__ uint32_t make_idesc_rt(int n, bool a_mn, bool b_mn) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn ? 1u : 0u) << 15) | ((b_mn ? 1u : 0u) << 16) |
+           ((uint32_t)(n >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+}
+// 16 consecutive f32 columns of this warp's 32 TMEM lanes.
+__device__ __forceinline__ void tc_ld16(uint32_t taddr, uint32_t (&r)[16]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr) : "memory");
+}
+// Barriers + tensor memory of `ncols` columns (a power of two >= 32), owned by warp 1.
+__device__ __forceinline__ void setup_cta(Barriers *bars, int warp, uint32_t ncols) {
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kMaxStages; ++s) { mbar_init(&bars->full[s], 1); mbar_init(&bars->empty[s], 1); }
+        mbar_init(&bars->acc_ready, 1);
+        bars->aborted = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(&bars->tmem_base)), "r"(ncols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+}
+__device__ __forceinline__ void teardown_cta(Barriers *bars, int warp, uint32_t ncols) {
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(bars->tmem_base), "r"(ncols) : "memory");
+    }
 }
 
 // SPLIT: the activation operand comes as two bf16 matrices (high part and remainder, whose sum
@@ -337,6 +377,198 @@ ffn_down_mma_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_con
     epilogue_done(t, warp);
 }
 
+
+// ---- decode batches of at most 128 tokens: weights on the M side -------------------------------
+// With few tokens the cheap orientation is the transposed one: the 128 channel rows of a weight
+// block are the MMA's M operand and the tokens its N columns (N = batch rounded up to 16), so an
+// instruction costs in proportion to the batch instead of a fixed 256 columns.
+//   gate/up:  D_g[128 ch, N] = W_gate[g rows] X^T,  D_u likewise;  actT[slot*128 + ch, token] = silu(D_g) D_u
+//   down:     D[128 out columns, N] = Wd_t[slice rows, 128 columns]^T actT[slice rows, tokens]
+// actT is stored channel-major (tokens contiguous, pitch 128), which makes it an N-major B operand for
+// the down GEMM; the Wd_t tile is the M-major A operand.
+template <bool SPLIT>
+__global__ void __launch_bounds__(kMmaThreads, 1)
+ffn_gateup_swap_kernel(const __grid_constant__ CUtensorMap tm_g, const __grid_constant__ CUtensorMap tm_u,
+                       const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_x_lo,
+                       const int32_t *__restrict__ glist, const int32_t *__restrict__ ng_dev, int N, int d,
+                       const uint32_t *__restrict__ gmask, __nv_bfloat16 *__restrict__ actT,
+                       __nv_bfloat16 *__restrict__ actT_lo, DeviceStatus *status) {
+    extern __shared__ uint8_t smem_raw[];
+    const int gi = blockIdx.x;
+    if (gi >= *ng_dev) return;
+    const int g = glist[gi];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    uint8_t *base = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    Barriers *bars = reinterpret_cast<Barriers *>(base + kRingBytesMma);
+    const int xbytes = N * 128;                                    // X tile: N tokens x 64 k
+    const int stage_bytes = 2 * kABytes + (SPLIT ? 2 : 1) * xbytes;
+    const int stages = min(6, kRingBytesMma / stage_bytes);
+    setup_cta(bars, warp, 256);
+    const int kblocks = d / BK;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            for (int kb = 0; kb < kblocks; ++kb) {
+                const int s = kb % stages;
+                if (kb >= stages && !mbar_wait(&bars->empty[s], ((kb / stages) - 1) & 1, bars, status)) break;
+                uint8_t *st = base + (size_t)s * stage_bytes;
+                mbar_expect_tx(&bars->full[s], stage_bytes);
+                tma_load_2d(st, &tm_g, kb * BK, g * 128, &bars->full[s]);
+                tma_load_2d(st + kABytes, &tm_u, kb * BK, g * 128, &bars->full[s]);
+                tma_load_2d(st + 2 * kABytes, &tm_x, kb * BK, 0, &bars->full[s]);
+                if (SPLIT) tma_load_2d(st + 2 * kABytes + xbytes, &tm_x_lo, kb * BK, 0, &bars->full[s]);
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            const uint32_t idesc = make_idesc_rt(N, false, false);
+            const uint32_t tmem = bars->tmem_base;
+            bool ok = true;
+            for (int kb = 0; kb < kblocks && ok; ++kb) {
+                const int s = kb % stages;
+                ok = mbar_wait(&bars->full[s], (kb / stages) & 1, bars, status);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t a_g = smem_u32(base + (size_t)s * stage_bytes), a_u = a_g + kABytes;
+                const uint32_t x0 = a_g + 2 * kABytes, x1 = x0 + xbytes;
+#pragma unroll
+                for (int k4 = 0; k4 < BK / 16; ++k4) {
+                    const uint64_t bd = desc_sw128(x0 + k4 * 32, 16), bl = desc_sw128(x1 + k4 * 32, 16);
+                    const uint64_t ag = desc_sw128(a_g + k4 * 32, 16), au = desc_sw128(a_u + k4 * 32, 16);
+                    tc_mma(tmem, ag, bd, idesc, (kb | k4) != 0);
+                    if (SPLIT) tc_mma(tmem, ag, bl, idesc, 1);
+                    tc_mma(tmem + 128, au, bd, idesc, (kb | k4) != 0);
+                    if (SPLIT) tc_mma(tmem + 128, au, bl, idesc, 1);
+                }
+                tc_commit(&bars->empty[s]);
+            }
+            if (ok) tc_commit(&bars->acc_ready);
+        }
+    } else {
+        const int q = warp & 3, ch = q * 32 + lane;
+        if (mbar_wait(&bars->acc_ready, 0, bars, status)) {
+            tc_fence_after();
+            const uint32_t tbase = bars->tmem_base + ((uint32_t)(q * 32) << 16);
+            const uint4 gm = *reinterpret_cast<const uint4 *>(gmask + (size_t)g * 4);
+            const uint32_t gw[4] = {gm.x, gm.y, gm.z, gm.w};
+            const size_t row = ((size_t)gi * 128 + ch) * 128;
+#pragma unroll 1
+            for (int c = 0; c < N / 16; ++c) {
+                uint32_t gv[16], uv[16];
+                tc_ld16(tbase + c * 16, gv);
+                tc_ld16(tbase + 128 + c * 16, uv);
+                tc_wait_ld();
+                const uint32_t bits = gw[(c * 16) >> 5] >> ((c * 16) & 31);
+                uint32_t hi[8], lo[8];
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const float k0 = (bits >> (2 * j)) & 1u ? 1.f : 0.f, k1 = (bits >> (2 * j + 1)) & 1u ? 1.f : 0.f;
+                    const float a0 = silu_f(__uint_as_float(gv[2 * j])) * __uint_as_float(uv[2 * j]) * k0;
+                    const float a1 = silu_f(__uint_as_float(gv[2 * j + 1])) * __uint_as_float(uv[2 * j + 1]) * k1;
+                    const __nv_bfloat162 p = __floats2bfloat162_rn(a0, a1);
+                    hi[j] = *reinterpret_cast<const uint32_t *>(&p);
+                    if (SPLIT) {
+                        const __nv_bfloat162 r = __floats2bfloat162_rn(a0 - __low2float(p), a1 - __high2float(p));
+                        lo[j] = *reinterpret_cast<const uint32_t *>(&r);
+                    }
+                }
+                uint4 *dst = reinterpret_cast<uint4 *>(actT + row + c * 16);
+                dst[0] = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+                dst[1] = make_uint4(hi[4], hi[5], hi[6], hi[7]);
+                if (SPLIT) {
+                    uint4 *dl = reinterpret_cast<uint4 *>(actT_lo + row + c * 16);
+                    dl[0] = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+                    dl[1] = make_uint4(lo[4], lo[5], lo[6], lo[7]);
+                }
+            }
+        }
+    }
+    teardown_cta(bars, warp, 256);
+}
+
+// grid (d / 128 output-column tiles, slices).  partial [slice][128 tokens][d].
+template <bool SPLIT>
+__global__ void __launch_bounds__(kMmaThreads, 1)
+ffn_down_swap_kernel(const __grid_constant__ CUtensorMap tm_wd, const __grid_constant__ CUtensorMap tm_act,
+                     const __grid_constant__ CUtensorMap tm_act_lo, const int32_t *__restrict__ glist,
+                     const int32_t *__restrict__ ng_dev, int N, int B, int d, float *__restrict__ partial,
+                     DeviceStatus *status) {
+    extern __shared__ uint8_t smem_raw[];
+    const int c0 = blockIdx.x * 128, z = blockIdx.y, Z = gridDim.y;
+    const int ng = *ng_dev;
+    const int gi0 = (int)(((long long)ng * z) / Z), gi1 = (int)(((long long)ng * (z + 1)) / Z);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    uint8_t *base = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    Barriers *bars = reinterpret_cast<Barriers *>(base + kRingBytesMma);
+    const int nblk = (N + 63) / 64;                                // token blocks of 64
+    const int bbytes = nblk * 64 * BK * 2;                         // actT tile: 64 k rows x tokens
+    const int stage_bytes = kABytes + (SPLIT ? 2 : 1) * bbytes;
+    const int stages = min(6, kRingBytesMma / stage_bytes);
+    setup_cta(bars, warp, 128);
+    const int kblocks = (gi1 - gi0) * 2;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            for (int kb = 0; kb < kblocks; ++kb) {
+                const int s = kb % stages;
+                if (kb >= stages && !mbar_wait(&bars->empty[s], ((kb / stages) - 1) & 1, bars, status)) break;
+                const int gi = gi0 + (kb >> 1), half = kb & 1;
+                const int wrow = glist[gi] * 128 + half * BK, arow = gi * 128 + half * BK;
+                uint8_t *st = base + (size_t)s * stage_bytes;
+                mbar_expect_tx(&bars->full[s], stage_bytes);
+                tma_load_2d(st, &tm_wd, c0, wrow, &bars->full[s]);
+                tma_load_2d(st + 64 * BK * 2, &tm_wd, c0 + 64, wrow, &bars->full[s]);
+                for (int i = 0; i < nblk; ++i) {
+                    tma_load_2d(st + kABytes + i * (64 * BK * 2), &tm_act, i * 64, arow, &bars->full[s]);
+                    if (SPLIT) tma_load_2d(st + kABytes + bbytes + i * (64 * BK * 2), &tm_act_lo, i * 64, arow, &bars->full[s]);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0 && kblocks > 0) {
+            const uint32_t idesc = make_idesc_rt(N, true, true);
+            const uint32_t tmem = bars->tmem_base;
+            bool ok = true;
+            for (int kb = 0; kb < kblocks && ok; ++kb) {
+                const int s = kb % stages;
+                ok = mbar_wait(&bars->full[s], (kb / stages) & 1, bars, status);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t a0 = smem_u32(base + (size_t)s * stage_bytes), b0 = a0 + kABytes, b1 = b0 + bbytes;
+#pragma unroll
+                for (int k4 = 0; k4 < BK / 16; ++k4) {
+                    const uint64_t ad = desc_sw128(a0 + k4 * 2048, 64 * BK * 2);
+                    tc_mma(tmem, ad, desc_sw128(b0 + k4 * 2048, 64 * BK * 2), idesc, (kb | k4) != 0);
+                    if (SPLIT) tc_mma(tmem, ad, desc_sw128(b1 + k4 * 2048, 64 * BK * 2), idesc, 1);
+                }
+                tc_commit(&bars->empty[s]);
+            }
+            if (ok) tc_commit(&bars->acc_ready);
+        }
+    } else {
+        const int q = warp & 3, col = c0 + q * 32 + lane;
+        float *dst = partial + (size_t)z * 128 * d + col;
+        if (kblocks == 0) {
+            for (int tkn = 0; tkn < B; ++tkn) dst[(size_t)tkn * d] = 0.f;
+        } else if (mbar_wait(&bars->acc_ready, 0, bars, status)) {
+            tc_fence_after();
+            const uint32_t tbase = bars->tmem_base + ((uint32_t)(q * 32) << 16);
+#pragma unroll 1
+            for (int c = 0; c < N / 16; ++c) {
+                uint32_t v[16];
+                tc_ld16(tbase + c * 16, v);
+                tc_wait_ld();
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                    const int tkn = c * 16 + j;
+                    if (tkn < B) dst[(size_t)tkn * d] = __uint_as_float(v[j]);
+                }
+            }
+        }
+    }
+    teardown_cta(bars, warp, 128);
+}
+
 // out[m, :] = residual[m, :] + sum_z partial[z, m, :], slices added in index order.
 template <typename OutT>
 __global__ void reduce_slices_kernel(const float *__restrict__ partial, int Z, int M, int m_pad, int d,
@@ -383,8 +615,8 @@ __global__ void split_bf16_kernel(const float *__restrict__ x, __nv_bfloat16 *__
 // ascending), *nu = their number.
 __global__ void __launch_bounds__(1024)
 bucket_kernel(const int32_t *__restrict__ support, int B, int k, int G, uint32_t *__restrict__ mask,
-              int32_t *__restrict__ counts, int32_t *__restrict__ offsets, int32_t *__restrict__ token_ids,
-              int32_t *__restrict__ glist, int32_t *__restrict__ nu) {
+              uint32_t *__restrict__ gmask, int32_t *__restrict__ counts, int32_t *__restrict__ offsets,
+              int32_t *__restrict__ token_ids, int32_t *__restrict__ glist, int32_t *__restrict__ nu) {
     __shared__ int cnt_s[kMaxG];
     __shared__ int off_s[kMaxG + 1];
     const int tid = threadIdx.x;
@@ -417,8 +649,13 @@ bucket_kernel(const int32_t *__restrict__ support, int B, int k, int G, uint32_t
     __syncthreads();
     if (tid < G) {
         int o = off_s[tid];
+        uint32_t w[4] = {0u, 0u, 0u, 0u};   // gmask: bit t of group tid, for the first 128 tokens
         for (int t = 0; t < B; ++t)
-            if ((mask[(size_t)t * 4 + (tid >> 5)] >> (tid & 31)) & 1u) token_ids[o++] = t;
+            if ((mask[(size_t)t * 4 + (tid >> 5)] >> (tid & 31)) & 1u) {
+                token_ids[o++] = t;
+                if (t < 128) w[t >> 5] |= 1u << (t & 31);
+            }
+        *reinterpret_cast<uint4 *>(gmask + (size_t)tid * 4) = make_uint4(w[0], w[1], w[2], w[3]);
     }
 }
 
@@ -461,12 +698,14 @@ cs_status prepare_ffn_mma(cs_plan *plan) {
     CS_CUDA_TRY(plan, cudaFuncSetAttribute(ffn_gateup_mma_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMmaSmem));
     CS_CUDA_TRY(plan, cudaFuncSetAttribute(ffn_down_mma_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMmaSmem));
     CS_CUDA_TRY(plan, cudaFuncSetAttribute(ffn_down_mma_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMmaSmem));
+    CS_CUDA_TRY(plan, cudaFuncSetAttribute(ffn_gateup_swap_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMmaSmem));
+    CS_CUDA_TRY(plan, cudaFuncSetAttribute(ffn_down_swap_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMmaSmem));
     return CS_OK;
 }
 
 cs_status launch_bucket(cs_plan *plan, const int32_t *support, int B, cudaStream_t st, int32_t *counts,
                         int32_t *offsets, int32_t *token_ids) {
-    bucket_kernel<<<1, 1024, 0, st>>>(support, B, plan->cfg.k, plan->G, plan->mask,
+    bucket_kernel<<<1, 1024, 0, st>>>(support, B, plan->cfg.k, plan->G, plan->mask, plan->gmask,
                                       counts ? counts : plan->counts, offsets ? offsets : plan->offsets,
                                       token_ids ? token_ids : plan->token_ids, plan->glist, plan->nu);
     plan->launches++;
@@ -527,6 +766,43 @@ cs_status launch_ffn_mma(cs_plan *plan, const cs_layer *L, const void *X, const 
         else
             reduce_slices_kernel<__nv_bfloat16><<<blocks, 256, 0, st>>>(plan->mma_partial, plan->last_slices, M, m_pad, c.d,
                                                                        residual, static_cast<__nv_bfloat16 *>(out_bf16));
+        plan->launches++;
+        CS_CUDA_TRY(plan, cudaGetLastError());
+    }
+    return CS_OK;
+}
+
+
+// Decode batches of 16..128 tokens (split-precision activations, union list and masks on the device).
+cs_status launch_ffn_mma_decode(cs_plan *plan, const cs_layer *L, const void *X, const void *X_lo, int B,
+                                const float *residual, float *out, cudaStream_t st) {
+    const cs_config &c = plan->cfg;
+    const int N = (B + 15) / 16 * 16;
+    __nv_bfloat16 *actT = static_cast<__nv_bfloat16 *>(plan->act);
+    __nv_bfloat16 *actT_lo = actT + (size_t)plan->G * 128 * 128;
+    CUtensorMap tm_g, tm_u, tm_x, tm_x_lo, tm_wd, tm_act, tm_act_lo;
+    if (!make_map(&tm_g, L->W_gate, c.d, c.d_ff, c.d, 128) || !make_map(&tm_u, L->W_up, c.d, c.d_ff, c.d, 128) ||
+        !make_map(&tm_x, X, c.d, B, c.d, N) || !make_map(&tm_x_lo, X_lo, c.d, B, c.d, N) ||
+        !make_map(&tm_wd, L->Wd_t, c.d, c.d_ff, c.d, BK) ||
+        !make_map(&tm_act, actT, 128, (uint64_t)plan->G * 128, 128, BK) ||
+        !make_map(&tm_act_lo, actT_lo, 128, (uint64_t)plan->G * 128, 128, BK))
+        return record_cuda(plan, cudaErrorInvalidValue, "cuTensorMapEncodeTiled");
+    const int Z = max(1, min(plan->sm_count / (c.d / 128), 8));
+    {
+        StageTimer timer(plan, CS_STAGE_EXEC, st);
+        ffn_gateup_swap_kernel<true><<<plan->G, kMmaThreads, kMmaSmem, st>>>(
+            tm_g, tm_u, tm_x, tm_x_lo, plan->glist, plan->nu, N, c.d, plan->gmask, actT, actT_lo, plan->status);
+        plan->launches++;
+        CS_CUDA_TRY(plan, cudaGetLastError());
+        ffn_down_swap_kernel<true><<<dim3(c.d / 128, Z), kMmaThreads, kMmaSmem, st>>>(
+            tm_wd, tm_act, tm_act_lo, plan->glist, plan->nu, N, B, c.d, plan->mma_partial, plan->status);
+        plan->launches++;
+        CS_CUDA_TRY(plan, cudaGetLastError());
+    }
+    {
+        StageTimer timer(plan, CS_STAGE_REDUCE, st);
+        const size_t total4 = (size_t)B * c.d / 4;
+        reduce_slices_kernel<float><<<(int)((total4 + 255) / 256), 256, 0, st>>>(plan->mma_partial, Z, B, 128, c.d, residual, out);
         plan->launches++;
         CS_CUDA_TRY(plan, cudaGetLastError());
     }
