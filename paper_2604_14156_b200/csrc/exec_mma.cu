@@ -403,7 +403,9 @@ ffn_gateup_swap_kernel(const __grid_constant__ CUtensorMap tm_g, const __grid_co
     const int xbytes = N * 128;                                    // X tile: N tokens x 64 k
     const int stage_bytes = 2 * kABytes + (SPLIT ? 2 : 1) * xbytes;
     const int stages = min(6, kRingBytesMma / stage_bytes);
-    setup_cta(bars, warp, 256);
+    const int NB = (SPLIT ? 2 : 1) * N;                            // columns per accumulator
+    const uint32_t tcols = 2 * NB <= 256 ? 256u : 512u;
+    setup_cta(bars, warp, tcols);
     const int kblocks = d / BK;
 
     if (warp == 0) {
@@ -421,7 +423,7 @@ ffn_gateup_swap_kernel(const __grid_constant__ CUtensorMap tm_g, const __grid_co
         }
     } else if (warp == 1) {
         if (lane == 0) {
-            const uint32_t idesc = make_idesc_rt(N, false, false);
+            const uint32_t idesc = make_idesc_rt(NB, false, false);
             const uint32_t tmem = bars->tmem_base;
             bool ok = true;
             for (int kb = 0; kb < kblocks && ok; ++kb) {
@@ -430,15 +432,14 @@ ffn_gateup_swap_kernel(const __grid_constant__ CUtensorMap tm_g, const __grid_co
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t a_g = smem_u32(base + (size_t)s * stage_bytes), a_u = a_g + kABytes;
-                const uint32_t x0 = a_g + 2 * kABytes, x1 = x0 + xbytes;
+                const uint32_t x0 = a_g + 2 * kABytes;
 #pragma unroll
                 for (int k4 = 0; k4 < BK / 16; ++k4) {
-                    const uint64_t bd = desc_sw128(x0 + k4 * 32, 16), bl = desc_sw128(x1 + k4 * 32, 16);
-                    const uint64_t ag = desc_sw128(a_g + k4 * 32, 16), au = desc_sw128(a_u + k4 * 32, 16);
-                    tc_mma(tmem, ag, bd, idesc, (kb | k4) != 0);
-                    if (SPLIT) tc_mma(tmem, ag, bl, idesc, 1);
-                    tc_mma(tmem + 128, au, bd, idesc, (kb | k4) != 0);
-                    if (SPLIT) tc_mma(tmem + 128, au, bl, idesc, 1);
+                    // x_hi and x_lo tiles are adjacent: one B operand of NB rows gives W x_hi in the first
+                    // N columns and W x_lo in the next N, at the cost of a single instruction
+                    const uint64_t bd = desc_sw128(x0 + k4 * 32, 16);
+                    tc_mma(tmem, desc_sw128(a_g + k4 * 32, 16), bd, idesc, (kb | k4) != 0);
+                    tc_mma(tmem + NB, desc_sw128(a_u + k4 * 32, 16), bd, idesc, (kb | k4) != 0);
                 }
                 tc_commit(&bars->empty[s]);
             }
@@ -456,8 +457,20 @@ ffn_gateup_swap_kernel(const __grid_constant__ CUtensorMap tm_g, const __grid_co
             for (int c = 0; c < N / 16; ++c) {
                 uint32_t gv[16], uv[16];
                 tc_ld16(tbase + c * 16, gv);
-                tc_ld16(tbase + 128 + c * 16, uv);
-                tc_wait_ld();
+                tc_ld16(tbase + NB + c * 16, uv);
+                if (SPLIT) {   // add the x_lo halves
+                    uint32_t g2[16], u2[16];
+                    tc_ld16(tbase + N + c * 16, g2);
+                    tc_ld16(tbase + NB + N + c * 16, u2);
+                    tc_wait_ld();
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) {
+                        gv[j] = __float_as_uint(__uint_as_float(gv[j]) + __uint_as_float(g2[j]));
+                        uv[j] = __float_as_uint(__uint_as_float(uv[j]) + __uint_as_float(u2[j]));
+                    }
+                } else {
+                    tc_wait_ld();
+                }
                 const uint32_t bits = gw[(c * 16) >> 5] >> ((c * 16) & 31);
                 uint32_t hi[8], lo[8];
 #pragma unroll
@@ -483,7 +496,7 @@ ffn_gateup_swap_kernel(const __grid_constant__ CUtensorMap tm_g, const __grid_co
             }
         }
     }
-    teardown_cta(bars, warp, 256);
+    teardown_cta(bars, warp, tcols);
 }
 
 // grid (d / 128 output-column tiles, slices).  partial [slice][128 tokens][d].
@@ -504,7 +517,9 @@ ffn_down_swap_kernel(const __grid_constant__ CUtensorMap tm_wd, const __grid_con
     const int bbytes = nblk * 64 * BK * 2;                         // actT tile: 64 k rows x tokens
     const int stage_bytes = kABytes + (SPLIT ? 2 : 1) * bbytes;
     const int stages = min(6, kRingBytesMma / stage_bytes);
-    setup_cta(bars, warp, 128);
+    const int NB = SPLIT ? 2 * nblk * 64 : N;                      // MMA columns: value blocks then remainder blocks
+    const uint32_t tcols = NB <= 128 ? 128u : 256u;
+    setup_cta(bars, warp, tcols);
     const int kblocks = (gi1 - gi0) * 2;
 
     if (warp == 0) {
@@ -526,7 +541,7 @@ ffn_down_swap_kernel(const __grid_constant__ CUtensorMap tm_wd, const __grid_con
         }
     } else if (warp == 1) {
         if (lane == 0 && kblocks > 0) {
-            const uint32_t idesc = make_idesc_rt(N, true, true);
+            const uint32_t idesc = make_idesc_rt(NB, true, true);
             const uint32_t tmem = bars->tmem_base;
             bool ok = true;
             for (int kb = 0; kb < kblocks && ok; ++kb) {
@@ -534,13 +549,11 @@ ffn_down_swap_kernel(const __grid_constant__ CUtensorMap tm_wd, const __grid_con
                 ok = mbar_wait(&bars->full[s], (kb / stages) & 1, bars, status);
                 if (!ok) break;
                 tc_fence_after();
-                const uint32_t a0 = smem_u32(base + (size_t)s * stage_bytes), b0 = a0 + kABytes, b1 = b0 + bbytes;
+                const uint32_t a0 = smem_u32(base + (size_t)s * stage_bytes), b0 = a0 + kABytes;
 #pragma unroll
-                for (int k4 = 0; k4 < BK / 16; ++k4) {
-                    const uint64_t ad = desc_sw128(a0 + k4 * 2048, 64 * BK * 2);
-                    tc_mma(tmem, ad, desc_sw128(b0 + k4 * 2048, 64 * BK * 2), idesc, (kb | k4) != 0);
-                    if (SPLIT) tc_mma(tmem, ad, desc_sw128(b1 + k4 * 2048, 64 * BK * 2), idesc, 1);
-                }
+                for (int k4 = 0; k4 < BK / 16; ++k4)   // remainder blocks follow the value blocks: one operand
+                    tc_mma(tmem, desc_sw128(a0 + k4 * 2048, 64 * BK * 2), desc_sw128(b0 + k4 * 2048, 64 * BK * 2),
+                           idesc, (kb | k4) != 0);
                 tc_commit(&bars->empty[s]);
             }
             if (ok) tc_commit(&bars->acc_ready);
@@ -557,7 +570,15 @@ ffn_down_swap_kernel(const __grid_constant__ CUtensorMap tm_wd, const __grid_con
             for (int c = 0; c < N / 16; ++c) {
                 uint32_t v[16];
                 tc_ld16(tbase + c * 16, v);
-                tc_wait_ld();
+                if (SPLIT) {
+                    uint32_t v2[16];
+                    tc_ld16(tbase + nblk * 64 + c * 16, v2);
+                    tc_wait_ld();
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) v[j] = __float_as_uint(__uint_as_float(v[j]) + __uint_as_float(v2[j]));
+                } else {
+                    tc_wait_ld();
+                }
 #pragma unroll
                 for (int j = 0; j < 16; ++j) {
                     const int tkn = c * 16 + j;
@@ -566,7 +587,7 @@ ffn_down_swap_kernel(const __grid_constant__ CUtensorMap tm_wd, const __grid_con
             }
         }
     }
-    teardown_cta(bars, warp, 128);
+    teardown_cta(bars, warp, tcols);
 }
 
 // out[m, :] = residual[m, :] + sum_z partial[z, m, :], slices added in index order.
