@@ -634,50 +634,88 @@ __global__ void split_bf16_kernel(const float *__restrict__ x, __nv_bfloat16 *__
 // One CTA.  mask [B][4] (bit g of token t), counts [G], offsets [G+1], token_ids [B*k] (tokens of
 // group g ascending at offsets[g]..offsets[g+1]), glist [G] (groups with a non-empty bucket,
 // ascending), *nu = their number.
+constexpr int kBucketSmemTokens = 2048;   // masks of this many tokens are kept in shared memory
+
 __global__ void __launch_bounds__(1024)
 bucket_kernel(const int32_t *__restrict__ support, int B, int k, int G, uint32_t *__restrict__ mask,
               uint32_t *__restrict__ gmask, int32_t *__restrict__ counts, int32_t *__restrict__ offsets,
               int32_t *__restrict__ token_ids, int32_t *__restrict__ glist, int32_t *__restrict__ nu) {
-    __shared__ int cnt_s[kMaxG];
-    __shared__ int off_s[kMaxG + 1];
-    const int tid = threadIdx.x;
-    if (tid < kMaxG) cnt_s[tid] = 0;
+    extern __shared__ uint32_t mask_s[];            // [min(B, kBucketSmemTokens)][4]
+    __shared__ int warp_tot[kMaxG / 32], warp_used[kMaxG / 32];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int Bs = min(B, kBucketSmemTokens);
+    // membership masks: one (token, slot) pair per thread, OR-ed into shared memory (tokens beyond
+    // the shared table go straight to global memory)
+    for (int i = tid; i < Bs * 4; i += blockDim.x) mask_s[i] = 0u;
+    for (int i = Bs * 4 + tid; i < B * 4; i += blockDim.x) mask[i] = 0u;
     __syncthreads();
-    for (int t = tid; t < B; t += blockDim.x) {
-        uint32_t w[4] = {0u, 0u, 0u, 0u};
-        for (int c = 0; c < k; ++c) {
-            const int g = support[(size_t)t * k + c];
-            if (g >= 0 && g < G) { w[g >> 5] |= 1u << (g & 31); atomicAdd(&cnt_s[g], 1); }
+    for (int i = tid; i < B * k; i += blockDim.x) {
+        const int t = i / k;
+        const int g = support[i];
+        if (g >= 0 && g < G) {
+            if (t < Bs) atomicOr(&mask_s[(size_t)t * 4 + (g >> 5)], 1u << (g & 31));
+            else atomicOr(&mask[(size_t)t * 4 + (g >> 5)], 1u << (g & 31));
         }
-        *reinterpret_cast<uint4 *>(mask + (size_t)t * 4) = make_uint4(w[0], w[1], w[2], w[3]);
     }
     __syncthreads();
-    if (tid == 0) {
-        int run = 0, n = 0;
-        for (int g = 0; g < G; ++g) {
-            off_s[g] = run; run += cnt_s[g];
-            if (cnt_s[g] > 0) glist[n++] = g;
-        }
-        off_s[G] = run;
-        *nu = n;
-    }
-    __syncthreads();
-    if (tid < G) { counts[tid] = cnt_s[tid]; offsets[tid] = off_s[tid]; }
-    if (tid == 0) offsets[G] = off_s[G];
-    // token lists in ascending token order: thread g walks the tokens (the masks were just written
-    // by this CTA; make them visible first)
+    for (int i = tid; i < Bs * 4; i += blockDim.x) mask[i] = mask_s[i];
     __threadfence_block();
     __syncthreads();
-    if (tid < G) {
-        int o = off_s[tid];
-        uint32_t w[4] = {0u, 0u, 0u, 0u};   // gmask: bit t of group tid, for the first 128 tokens
-        for (int t = 0; t < B; ++t)
-            if ((mask[(size_t)t * 4 + (tid >> 5)] >> (tid & 31)) & 1u) {
-                token_ids[o++] = t;
-                if (t < 128) w[t >> 5] |= 1u << (t & 31);
+    if (tid >= kMaxG) return;   // one thread per group from here on (warps 0..3)
+    const int g = tid;
+    const int word = g >> 5;
+    const uint32_t bit = 1u << (g & 31);
+    auto member = [&](int t) -> bool {
+        return ((t < Bs ? mask_s[(size_t)t * 4 + word] : mask[(size_t)t * 4 + word]) & bit) != 0u;
+    };
+    // the transposed mask (bit t of group g) for the first 128 tokens, in four scalar words, and the
+    // bucket size
+    uint32_t w0 = 0u, w1 = 0u, w2 = 0u, w3 = 0u;
+    int cnt = 0;
+    if (g < G) {
+        const int sh = g & 31;
+        auto gather32 = [&](int t0) -> uint32_t {
+            uint32_t wd = 0u;
+#pragma unroll 8
+            for (int tt = 0; tt < 32; ++tt) {
+                const int t = t0 + tt;
+                if (t < Bs) wd |= ((mask_s[(size_t)t * 4 + word] >> sh) & 1u) << tt;
             }
-        *reinterpret_cast<uint4 *>(gmask + (size_t)tid * 4) = make_uint4(w[0], w[1], w[2], w[3]);
+            return wd;
+        };
+        w0 = gather32(0);
+        if (B > 32) w1 = gather32(32);
+        if (B > 64) w2 = gather32(64);
+        if (B > 96) w3 = gather32(96);
+        cnt = __popc(w0) + __popc(w1) + __popc(w2) + __popc(w3);
+        for (int t = 128; t < B; ++t) cnt += member(t);
     }
+    // exclusive prefix sums over groups of the bucket sizes and of the non-empty flags
+    int inc = cnt, used = cnt > 0, uinc = used;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int a = __shfl_up_sync(0xffffffffu, inc, o), b = __shfl_up_sync(0xffffffffu, uinc, o);
+        if (lane >= o) { inc += a; uinc += b; }
+    }
+    if (lane == 31) { warp_tot[warp] = inc; warp_used[warp] = uinc; }
+    // only warps 0..3 are alive: a named barrier over their 128 threads
+    asm volatile("bar.sync 1, 128;" ::: "memory");
+    int off = inc - cnt, uoff = uinc - used;
+    for (int w2 = 0; w2 < warp; ++w2) { off += warp_tot[w2]; uoff += warp_used[w2]; }
+    if (g < G) {
+        counts[g] = cnt;
+        offsets[g] = off;
+        if (used) glist[uoff] = g;
+        *reinterpret_cast<uint4 *>(gmask + (size_t)g * 4) = make_uint4(w0, w1, w2, w3);
+        int o = off;   // tokens of the bucket in ascending order: walk the set bits, then the tail
+        auto emit = [&](uint32_t wd, int t0) {
+            while (wd) { token_ids[o++] = t0 + __ffs(wd) - 1; wd &= wd - 1; }
+        };
+        emit(w0, 0); emit(w1, 32); emit(w2, 64); emit(w3, 96);
+        for (int t = 128; t < B; ++t)
+            if (member(t)) token_ids[o++] = t;
+    }
+    if (g == kMaxG - 1) { offsets[G] = off + cnt; *nu = uoff + used; }
 }
 
 // ---- host side ----------------------------------------------------------------------------------
@@ -726,7 +764,8 @@ cs_status prepare_ffn_mma(cs_plan *plan) {
 
 cs_status launch_bucket(cs_plan *plan, const int32_t *support, int B, cudaStream_t st, int32_t *counts,
                         int32_t *offsets, int32_t *token_ids) {
-    bucket_kernel<<<1, 1024, 0, st>>>(support, B, plan->cfg.k, plan->G, plan->mask, plan->gmask,
+    const size_t smem = (size_t)min(B, kBucketSmemTokens) * 16;
+    bucket_kernel<<<1, 1024, smem, st>>>(support, B, plan->cfg.k, plan->G, plan->mask, plan->gmask,
                                       counts ? counts : plan->counts, offsets ? offsets : plan->offsets,
                                       token_ids ? token_ids : plan->token_ids, plan->glist, plan->nu);
     plan->launches++;
