@@ -106,6 +106,26 @@ cs_status launch_ffn_mma_decode(cs_plan *plan, const cs_layer *L, const void *X,
                                 const float *residual, float *out, cudaStream_t st);
 cs_status launch_prompt_mean(cs_plan *plan, const void *H, int n, float *hbar, cudaStream_t st);
 
+// Programmatic dependent launch: a kernel launched through launch_pdl may start while its
+// predecessor in the stream is still running (its CTAs become resident, run their prologue and
+// then block in pdl_wait until the predecessor's writes are complete and visible).  Kernels call
+// pdl_launch_dependents early so that their successor can do the same.  Both are no-ops for a
+// kernel launched the ordinary way.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                              Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 // ---- small device helpers -------------------------------------------------------------------
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll

@@ -68,6 +68,8 @@ ffn_gather_kernel(const WT *__restrict__ Wg, const WT *__restrict__ Wu, const WT
     const int chunks = d / E;                                       // chunks per row
     const int nseg = (chunks + kUnitChunks * 32 - 1) / (kUnitChunks * 32);
     const int nunits = nrows * nseg;
+    pdl_launch_dependents();
+    pdl_wait();   // supports and activations come from the kernels before
 
     if (tid < nrows) {
         const int c = r_begin + tid;
@@ -208,6 +210,8 @@ reduce_partials_kernel(const float *__restrict__ partial, int nx, int d, const f
     const int col = blockIdx.x * 32 + (threadIdx.x & 31);  // float4 column
     const int grp = threadIdx.x >> 5;
     const int cols = d >> 2;
+    pdl_launch_dependents();
+    pdl_wait();
     float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
     if (col < cols) {
         const float4 *src = reinterpret_cast<const float4 *>(partial + (size_t)t * nx * d) + col;
@@ -270,7 +274,7 @@ static void launch_gather_kernel(dim3 grid, cudaStream_t st, int cpt, int chunks
                                  float *partial) {
     const bool full = chunks % kGatherThreads == 0 && (cpt == 1 || cpt == 2 || cpt == 4);
 #define CS_GATHER_CASE(N, F)                                                                          \
-    ffn_gather_kernel<WT, N, F><<<grid, kGatherThreads, kRingBytes, st>>>(Wg, Wu, Wd, h, sup, d, b, k, partial)
+    launch_pdl(ffn_gather_kernel<WT, N, F>, grid, dim3(kGatherThreads), kRingBytes, st, Wg, Wu, Wd, h, sup, d, b, k, partial)
     if (cpt <= 1) { if (full) CS_GATHER_CASE(1, true); else CS_GATHER_CASE(1, false); }
     else if (cpt <= 2) { if (full) CS_GATHER_CASE(2, true); else CS_GATHER_CASE(2, false); }
     else { if (full) CS_GATHER_CASE(4, true); else CS_GATHER_CASE(4, false); }
@@ -303,8 +307,8 @@ static cs_status gather_typed(cs_plan *plan, const cs_layer *L, const float *h, 
         dim3 rgrid((c.d / 4 + 31) / 32, nb);
         {
             StageTimer timer(plan, CS_STAGE_REDUCE, st);
-            reduce_partials_kernel<<<rgrid, 32 * kReduceGroups, 0, st>>>(
-                plan->partial, nx, c.d, residual ? residual + (size_t)t0 * c.d : nullptr, out + (size_t)t0 * c.d);
+            launch_pdl(reduce_partials_kernel, rgrid, dim3(32 * kReduceGroups), 0, st, (const float *)plan->partial, nx,
+                       c.d, residual ? residual + (size_t)t0 * c.d : (const float *)nullptr, out + (size_t)t0 * c.d);
         }
         plan->launches++;
         CS_CUDA_TRY(plan, cudaGetLastError());

@@ -40,10 +40,12 @@ recover_kernel(const float *__restrict__ Phi, float mu, const float *__restrict_
     float *phi_s = smem + 4 * kMaxG + kRecMaxWarps * kMaxM + kRecMaxWarps;          // [m][Gp]
 
     const int t = blockIdx.x;
+    pdl_launch_dependents();
     for (int col = tid; col < G; col += blockDim.x) {
 #pragma unroll 8
         for (int row = 0; row < m; ++row) phi_s[row * Gp + col] = __ldg(Phi + row * G + col);
     }
+    pdl_wait();   // Phi is a parameter and was staged above; y comes from the sketch kernel
     float yv[ROWS];
 #pragma unroll
     for (int q = 0; q < ROWS; ++q) {
@@ -167,9 +169,9 @@ cs_status launch_recover(cs_plan *plan, const float *Phi, float mu, const float 
     const int warps = (G + 31) / 32;
     const size_t smem = sizeof(float) * ((size_t)c.m * (G | 1) + 4 * kMaxG + kRecMaxWarps * kMaxM + kRecMaxWarps);
     if (c.m <= 32)
-        recover_kernel<1><<<B, 32 * warps, smem, st>>>(Phi, mu, y, c.m, G, c.k, c.T, support, z, resid);
+        launch_pdl(recover_kernel<1>, dim3(B), dim3(32 * warps), smem, st, Phi, mu, y, c.m, G, c.k, c.T, support, z, resid);
     else
-        recover_kernel<2><<<B, 32 * warps, smem, st>>>(Phi, mu, y, c.m, G, c.k, c.T, support, z, resid);
+        launch_pdl(recover_kernel<2>, dim3(B), dim3(32 * warps), smem, st, Phi, mu, y, c.m, G, c.k, c.T, support, z, resid);
     plan->launches++;
     CS_CUDA_TRY(plan, cudaGetLastError());
     return CS_OK;

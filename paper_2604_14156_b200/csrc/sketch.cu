@@ -27,6 +27,8 @@ sketch_kernel(const float *__restrict__ S, const float *__restrict__ x, const fl
     const int nrows = min(rows_per_cta, m - r0);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int chunks = d >> 2;
+    pdl_launch_dependents();
+    pdl_wait();   // x may be the previous kernel's output
 
     float4 xv[CPT];
     float ss = 0.f;
@@ -93,7 +95,7 @@ cs_status launch_sketch(cs_plan *plan, const float *S, const float *x, const flo
     dim3 grid((c.m + rpc - 1) / rpc, B);
     const int cpt = (c.d / 4 + kSketchThreads - 1) / kSketchThreads;
 #define CS_SKETCH_CASE(N)                                                                            \
-    sketch_kernel<N><<<grid, kSketchThreads, 0, st>>>(S, x, gamma, c.rms_eps, c.m, c.d, rpc, y, n_out)
+    launch_pdl(sketch_kernel<N>, grid, dim3(kSketchThreads), 0, st, S, x, gamma, c.rms_eps, c.m, c.d, rpc, y, n_out)
     if (cpt <= 1) CS_SKETCH_CASE(1);
     else if (cpt <= 2) CS_SKETCH_CASE(2);
     else if (cpt <= 4) CS_SKETCH_CASE(4);
