@@ -200,7 +200,8 @@ cs_status cs_layer_step_host(cs_plan *plan, const cs_layer *layer, const float *
  * by CUDA events on the call's stream.  cs_plan_stage_times synchronises `stream` and returns the
  * device time in milliseconds of each stage's kernels in the most recent call that ran it.
  */
-enum { CS_STAGE_SKETCH = 0, CS_STAGE_RECOVER = 1, CS_STAGE_EXEC = 2, CS_STAGE_REDUCE = 3, CS_STAGE_COUNT = 4 };
+enum { CS_STAGE_SKETCH = 0, CS_STAGE_RECOVER = 1, CS_STAGE_EXEC = 2, CS_STAGE_REDUCE = 3,
+       CS_STAGE_EXEC2 = 4 /* down GEMM of the tensor-core decode path */, CS_STAGE_COUNT = 5 };
 cs_status cs_plan_enable_timing(cs_plan *plan, int32_t on);
 cs_status cs_plan_stage_times(cs_plan *plan, void *stream, float ms[CS_STAGE_COUNT]);
 

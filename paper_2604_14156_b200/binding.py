@@ -68,7 +68,7 @@ def load_library():
     lib.cs_ffn_exec_shared.argtypes = [vp, ctypes.POINTER(_Layer), vp, i32, vp, vp, vp]
     lib.cs_layer_step_host.argtypes = [vp, ctypes.POINTER(_Layer), vp, i32, vp, vp, vp]
     lib.cs_plan_enable_timing.argtypes = [vp, i32]
-    lib.cs_plan_stage_times.argtypes = [vp, vp, ctypes.POINTER(f32 * 4)]
+    lib.cs_plan_stage_times.argtypes = [vp, vp, ctypes.POINTER(f32 * 5)]
     lib.cs_ffn_exec_static.argtypes = [ctypes.POINTER(_Config), ctypes.POINTER(_Layer), vp, vp, i32, vp, vp, vp]
     lib.cs_ffn_exec_static.restype = ctypes.c_int
     lib.cs_bucket.argtypes = [vp, vp, i32, vp, vp, vp, vp]
@@ -142,8 +142,9 @@ class Plan:
         self.check(self.lib.cs_plan_enable_timing(self.handle, int(on)), "cs_plan_enable_timing")
 
     def stage_times(self, stream=None):
-        """Milliseconds of (sketch, recover, exec, reduce) in the most recent call."""
-        ms = (ctypes.c_float * 4)()
+        """Milliseconds of (sketch, recover, exec, reduce, exec2) in the most recent call; exec2 is
+        the down GEMM of the tensor-core decode path (0 otherwise)."""
+        ms = (ctypes.c_float * 5)()
         self.check(self.lib.cs_plan_stage_times(self.handle, _stream(stream), ctypes.byref(ms)),
                    "cs_plan_stage_times")
         return tuple(ms)

@@ -83,6 +83,9 @@ cs_status cs_plan_create(const cs_config *cfg, cs_plan **out) {
     alloc((void **)&p->x_host_out, nt * cfg->d * sizeof(float));
     for (int i = 0; i < 2 * CS_STAGE_COUNT; ++i)
         if (e == cudaSuccess) e = cudaEventCreate(&p->ev[i]);
+    if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&p->side, cudaStreamNonBlocking);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p->ev_fork, cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p->ev_join, cudaEventDisableTiming);
     if (e == cudaSuccess) e = cudaMemset(p->status, 0, sizeof(DeviceStatus));
     if (e == cudaSuccess && prepare_ffn_gather(p) != CS_OK) e = cudaErrorUnknown;
     if (e == cudaSuccess && p->mma_ok && prepare_ffn_mma(p) != CS_OK) e = cudaErrorUnknown;
@@ -103,6 +106,9 @@ cs_status cs_plan_destroy(cs_plan *p) {
     cudaFree(p->nu); cudaFree(p->x_bf16); cudaFree(p->act); cudaFree(p->mma_partial);
     for (int i = 0; i < 2 * CS_STAGE_COUNT; ++i)
         if (p->ev[i] != nullptr) cudaEventDestroy(p->ev[i]);
+    if (p->ev_fork != nullptr) cudaEventDestroy(p->ev_fork);
+    if (p->ev_join != nullptr) cudaEventDestroy(p->ev_join);
+    if (p->side != nullptr) cudaStreamDestroy(p->side);
     delete p;
     return CS_OK;
 }
@@ -128,19 +134,50 @@ static cs_status check_weights(const cs_layer *L) {
     return CS_OK;
 }
 
-// Large decode batches on the tensor cores: activations to bf16, buckets / masks / union list from
-// the supports, then the two grouped GEMMs over the union.
+extern "C++" {
+static bool use_decode_mma(const cs_plan *plan, int B) { return plan->mma_ok && B >= kMmaMinTokens && B <= 128; }
+
+// Tensor-core decode path for 16..128 tokens.  The gate/up GEMM needs no supports (at these batch
+// sizes the union of the supports is, to within a group or two, every group), so it runs on the
+// caller's stream while `side_work` -- sketch / recovery / bucketing -- runs on the plan's second
+// stream; the two join before the activations are masked and the down GEMM starts.
+template <typename SideWork>
+static cs_status exec_decode_overlapped(cs_plan *plan, const cs_layer *layer, const float *h, int B,
+                                        const float *residual, float *out, cudaStream_t st, SideWork side_work) {
+    __nv_bfloat16 *x_hi = static_cast<__nv_bfloat16 *>(plan->x_bf16);
+    __nv_bfloat16 *x_lo = x_hi + (size_t)plan->cfg.max_tokens * plan->cfg.d;
+    CS_CUDA_TRY(plan, cudaEventRecord(plan->ev_fork, st));
+    CS_CUDA_TRY(plan, cudaStreamWaitEvent(plan->side, plan->ev_fork, 0));
+    cs_status s = side_work(plan->side);
+    if (s != CS_OK) return s;
+    CS_CUDA_TRY(plan, cudaEventRecord(plan->ev_join, plan->side));
+    // f32 activations go in as two bf16 parts so that the result keeps f32-level accuracy
+    s = launch_split_bf16(plan, h, x_hi, x_lo, (size_t)B * plan->cfg.d, st);
+    if (s != CS_OK) return s;
+    s = launch_decode_gateup(plan, layer, x_hi, x_lo, B, false, st);
+    if (s != CS_OK) return s;
+    CS_CUDA_TRY(plan, cudaStreamWaitEvent(st, plan->ev_join, 0));
+    s = launch_decode_mask(plan, B, st);
+    if (s != CS_OK) return s;
+    return launch_decode_down(plan, layer, B, true, residual, out, st);
+}
+
+}  // extern "C++"
+
+// Dispatch of the actuator by batch size: gather GEMV, tensor-core decode path, or (more than 128
+// tokens) the token-tiled grouped GEMMs over the union list.
 static cs_status exec_dispatch(cs_plan *plan, const cs_layer *layer, const float *h, const int32_t *support,
                                int B, const float *residual, float *out, cudaStream_t st) {
     if (!plan->mma_ok || B < kMmaMinTokens) return launch_ffn_gather(plan, layer, h, support, B, residual, out, st);
-    // f32 activations go in as two bf16 parts so that the result keeps f32-level accuracy
+    if (use_decode_mma(plan, B))
+        return exec_decode_overlapped(plan, layer, h, B, residual, out, st,
+                                      [&](cudaStream_t side) { return launch_bucket(plan, support, B, side); });
     __nv_bfloat16 *x_hi = static_cast<__nv_bfloat16 *>(plan->x_bf16);
     __nv_bfloat16 *x_lo = x_hi + (size_t)plan->cfg.max_tokens * plan->cfg.d;
     cs_status s = launch_split_bf16(plan, h, x_hi, x_lo, (size_t)B * plan->cfg.d, st);
     if (s != CS_OK) return s;
     s = launch_bucket(plan, support, B, st);
     if (s != CS_OK) return s;
-    if (B <= 128) return launch_ffn_mma_decode(plan, layer, x_hi, x_lo, B, residual, out, st);
     return launch_ffn_mma(plan, layer, x_hi, x_lo, B, plan->glist, plan->nu, 0, plan->mask, residual, out, nullptr, st);
 }
 
@@ -183,6 +220,21 @@ cs_status cs_layer_step(cs_plan *plan, const cs_layer *layer, const float *x, in
     const bool norm = layer->rms_gamma != nullptr;
     const float *n = norm ? plan->n_buf : x;
     int32_t *sup = support_out != nullptr ? support_out : plan->sup_buf;
+    if (use_decode_mma(plan, B)) {
+        // recovery (and, without a normalisation to wait for, the sketch too) beside the gate/up GEMM
+        if (norm) {
+            s = launch_sketch(plan, layer->S, x, layer->rms_gamma, B, plan->y_buf, plan->n_buf, st);
+            if (s != CS_OK) return s;
+        }
+        return exec_decode_overlapped(plan, layer, n, B, layer->add_residual ? x : nullptr, x_out, st,
+                                      [&](cudaStream_t side) {
+            cs_status r = CS_OK;
+            if (!norm) r = launch_sketch(plan, layer->S, x, nullptr, B, plan->y_buf, nullptr, side);
+            if (r == CS_OK) r = launch_recover(plan, layer->Phi, layer->mu, plan->y_buf, B, sup, z_out, resid_out, side);
+            if (r == CS_OK) r = launch_bucket(plan, sup, B, side);
+            return r;
+        });
+    }
     s = launch_sketch(plan, layer->S, x, layer->rms_gamma, B, plan->y_buf, norm ? plan->n_buf : nullptr, st);
     if (s != CS_OK) return s;
     s = launch_recover(plan, layer->Phi, layer->mu, plan->y_buf, B, sup, z_out, resid_out, st);

@@ -57,6 +57,8 @@ struct cs_plan {
     float *x_host_in;  // [max_tokens, d] staging for the host-buffer entry point
     float *x_host_out; // [max_tokens, d]
     cudaEvent_t ev[2 * CS_STAGE_COUNT];  // start/stop per stage
+    cudaStream_t side;                   // second stream: recovery runs beside the gate/up GEMM
+    cudaEvent_t ev_fork, ev_join;
     int timing;
     int stage_seen[CS_STAGE_COUNT];
     int nx_max;
@@ -102,27 +104,33 @@ cs_status launch_split_bf16(cs_plan *plan, const float *x, void *y_hi, void *y_l
 cs_status launch_ffn_mma(cs_plan *plan, const cs_layer *L, const void *X, const void *X_lo, int M, const int32_t *glist,
                          const int32_t *ng_dev, int ng_host, const uint32_t *mask, const float *residual,
                          float *out_f32, void *out_bf16, cudaStream_t st);
-cs_status launch_ffn_mma_decode(cs_plan *plan, const cs_layer *L, const void *X, const void *X_lo, int B,
-                                const float *residual, float *out, cudaStream_t st);
+cs_status launch_decode_gateup(cs_plan *plan, const cs_layer *L, const void *X, const void *X_lo, int B,
+                               bool masked, cudaStream_t st);
+cs_status launch_decode_mask(cs_plan *plan, int B, cudaStream_t st);
+cs_status launch_decode_down(cs_plan *plan, const cs_layer *L, int B, bool act_by_group, const float *residual,
+                             float *out, cudaStream_t st);
 cs_status launch_prompt_mean(cs_plan *plan, const void *H, int n, float *hbar, cudaStream_t st);
 
 // Programmatic dependent launch: a kernel launched through launch_pdl may start while its
 // predecessor in the stream is still running (its CTAs become resident, run their prologue and
 // then block in pdl_wait until the predecessor's writes are complete and visible).  Kernels call
 // pdl_launch_dependents early so that their successor can do the same.  Both are no-ops for a
-// kernel launched the ordinary way.
+// kernel launched the ordinary way (pdl = false).  Only the small-batch chain uses it: its kernels are
+// a few microseconds long and launch latency matters; with the large tensor-core kernels early-resident
+// dependents measurably slowed the step down.
+inline bool pdl_for(const cs_plan *plan, int B) { return !(plan->mma_ok && B >= kMmaMinTokens); }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 template <typename... KArgs, typename... Args>
-inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
-                              Args... args) {
+inline cudaError_t launch_pdl(bool pdl, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
+                              cudaStream_t st, Args... args) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr; cfg.numAttrs = 1;
+    cfg.attrs = attr; cfg.numAttrs = pdl ? 1 : 0;
     return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }
 

@@ -274,7 +274,7 @@ static void launch_gather_kernel(dim3 grid, cudaStream_t st, int cpt, int chunks
                                  float *partial) {
     const bool full = chunks % kGatherThreads == 0 && (cpt == 1 || cpt == 2 || cpt == 4);
 #define CS_GATHER_CASE(N, F)                                                                          \
-    launch_pdl(ffn_gather_kernel<WT, N, F>, grid, dim3(kGatherThreads), kRingBytes, st, Wg, Wu, Wd, h, sup, d, b, k, partial)
+    launch_pdl(true, ffn_gather_kernel<WT, N, F>, grid, dim3(kGatherThreads), kRingBytes, st, Wg, Wu, Wd, h, sup, d, b, k, partial)
     if (cpt <= 1) { if (full) CS_GATHER_CASE(1, true); else CS_GATHER_CASE(1, false); }
     else if (cpt <= 2) { if (full) CS_GATHER_CASE(2, true); else CS_GATHER_CASE(2, false); }
     else { if (full) CS_GATHER_CASE(4, true); else CS_GATHER_CASE(4, false); }
@@ -307,7 +307,7 @@ static cs_status gather_typed(cs_plan *plan, const cs_layer *L, const float *h, 
         dim3 rgrid((c.d / 4 + 31) / 32, nb);
         {
             StageTimer timer(plan, CS_STAGE_REDUCE, st);
-            launch_pdl(reduce_partials_kernel, rgrid, dim3(32 * kReduceGroups), 0, st, (const float *)plan->partial, nx,
+            launch_pdl(true, reduce_partials_kernel, rgrid, dim3(32 * kReduceGroups), 0, st, (const float *)plan->partial, nx,
                        c.d, residual ? residual + (size_t)t0 * c.d : (const float *)nullptr, out + (size_t)t0 * c.d);
         }
         plan->launches++;

@@ -394,9 +394,12 @@ ffn_gateup_swap_kernel(const __grid_constant__ CUtensorMap tm_g, const __grid_co
                        const uint32_t *__restrict__ gmask, __nv_bfloat16 *__restrict__ actT,
                        __nv_bfloat16 *__restrict__ actT_lo, DeviceStatus *status) {
     extern __shared__ uint8_t smem_raw[];
+    // glist == NULL: one CTA per group of the layer, activations stored at the group's own index and
+    // left unmasked (the supports are still being recovered on another stream; mask_act_kernel
+    // applies them afterwards).
     const int gi = blockIdx.x;
-    if (gi >= *ng_dev) return;
-    const int g = glist[gi];
+    if (glist != nullptr && gi >= *ng_dev) return;
+    const int g = glist != nullptr ? glist[gi] : gi;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     uint8_t *base = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     Barriers *bars = reinterpret_cast<Barriers *>(base + kRingBytesMma);
@@ -450,7 +453,8 @@ ffn_gateup_swap_kernel(const __grid_constant__ CUtensorMap tm_g, const __grid_co
         if (mbar_wait(&bars->acc_ready, 0, bars, status)) {
             tc_fence_after();
             const uint32_t tbase = bars->tmem_base + ((uint32_t)(q * 32) << 16);
-            const uint4 gm = *reinterpret_cast<const uint4 *>(gmask + (size_t)g * 4);
+            const uint4 gm = gmask != nullptr ? *reinterpret_cast<const uint4 *>(gmask + (size_t)g * 4)
+                                              : make_uint4(~0u, ~0u, ~0u, ~0u);
             const uint32_t gw[4] = {gm.x, gm.y, gm.z, gm.w};
             const size_t row = ((size_t)gi * 128 + ch) * 128;
 #pragma unroll 1
@@ -504,8 +508,8 @@ template <bool SPLIT>
 __global__ void __launch_bounds__(kMmaThreads, 1)
 ffn_down_swap_kernel(const __grid_constant__ CUtensorMap tm_wd, const __grid_constant__ CUtensorMap tm_act,
                      const __grid_constant__ CUtensorMap tm_act_lo, const int32_t *__restrict__ glist,
-                     const int32_t *__restrict__ ng_dev, int N, int B, int d, float *__restrict__ partial,
-                     DeviceStatus *status) {
+                     const int32_t *__restrict__ ng_dev, int N, int B, int d, int act_by_group,
+                     float *__restrict__ partial, DeviceStatus *status) {
     extern __shared__ uint8_t smem_raw[];
     const int c0 = blockIdx.x * 128, z = blockIdx.y, Z = gridDim.y;
     const int ng = *ng_dev;
@@ -528,7 +532,8 @@ ffn_down_swap_kernel(const __grid_constant__ CUtensorMap tm_wd, const __grid_con
                 const int s = kb % stages;
                 if (kb >= stages && !mbar_wait(&bars->empty[s], ((kb / stages) - 1) & 1, bars, status)) break;
                 const int gi = gi0 + (kb >> 1), half = kb & 1;
-                const int wrow = glist[gi] * 128 + half * BK, arow = gi * 128 + half * BK;
+                const int wrow = glist[gi] * 128 + half * BK;
+                const int arow = (act_by_group ? glist[gi] : gi) * 128 + half * BK;
                 uint8_t *st = base + (size_t)s * stage_bytes;
                 mbar_expect_tx(&bars->full[s], stage_bytes);
                 tma_load_2d(st, &tm_wd, c0, wrow, &bars->full[s]);
@@ -588,6 +593,28 @@ ffn_down_swap_kernel(const __grid_constant__ CUtensorMap tm_wd, const __grid_con
         }
     }
     teardown_cta(bars, warp, tcols);
+}
+
+
+// Zeroes the activations of (group, token) pairs outside the supports: row r of actT belongs to
+// group r / 128; bit t of gmask[group] says whether token t owns the group.  One thread per row
+// and 8-token chunk, for the value and the remainder matrix.
+__global__ void mask_act_kernel(__nv_bfloat16 *__restrict__ actT, __nv_bfloat16 *__restrict__ actT_lo,
+                                const uint32_t *__restrict__ gmask, int rows, int N) {
+    const int chunks = N / 8;
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= rows * chunks) return;
+    const int r = i / chunks, c = i - r * chunks;
+    const uint32_t bits = (gmask[(size_t)(r >> 7) * 4 + ((c * 8) >> 5)] >> ((c * 8) & 31)) & 0xffu;
+    if (bits == 0xffu) return;
+    const uint32_t m0 = (bits & 1u ? 0xffffu : 0u) | (bits & 2u ? 0xffff0000u : 0u);
+    const uint32_t m1 = (bits & 4u ? 0xffffu : 0u) | (bits & 8u ? 0xffff0000u : 0u);
+    const uint32_t m2 = (bits & 16u ? 0xffffu : 0u) | (bits & 32u ? 0xffff0000u : 0u);
+    const uint32_t m3 = (bits & 64u ? 0xffffu : 0u) | (bits & 128u ? 0xffff0000u : 0u);
+    uint4 *p = reinterpret_cast<uint4 *>(actT + (size_t)r * 128 + c * 8);
+    uint4 v = *p; v.x &= m0; v.y &= m1; v.z &= m2; v.w &= m3; *p = v;
+    uint4 *q = reinterpret_cast<uint4 *>(actT_lo + (size_t)r * 128 + c * 8);
+    uint4 w = *q; w.x &= m0; w.y &= m1; w.z &= m2; w.w &= m3; *q = w;
 }
 
 // out[m, :] = residual[m, :] + sum_z partial[z, m, :], slices added in index order.
@@ -833,29 +860,64 @@ cs_status launch_ffn_mma(cs_plan *plan, const cs_layer *L, const void *X, const 
 }
 
 
-// Decode batches of 16..128 tokens (split-precision activations, union list and masks on the device).
-cs_status launch_ffn_mma_decode(cs_plan *plan, const cs_layer *L, const void *X, const void *X_lo, int B,
-                                const float *residual, float *out, cudaStream_t st) {
+// Decode batches of 16..128 tokens in three launches that the caller orders (the gate/up GEMM can
+// run while the supports are still being recovered on another stream):
+//   launch_decode_gateup(masked = false)  every group of the layer, activations unmasked, stored at the
+//                                         group's own index;   (masked = true: union list + masks)
+//   launch_decode_mask                    zeroes the (group, token) pairs outside the supports
+//   launch_decode_down                    down GEMM over the union list, slice reduction, residual
+static bool decode_maps(cs_plan *plan, const cs_layer *L, const void *X, const void *X_lo, int B, int N,
+                        CUtensorMap *tm) {
+    const cs_config &c = plan->cfg;
+    __nv_bfloat16 *actT = static_cast<__nv_bfloat16 *>(plan->act);
+    __nv_bfloat16 *actT_lo = actT + (size_t)plan->G * 128 * 128;
+    return make_map(&tm[0], L->W_gate, c.d, c.d_ff, c.d, 128) && make_map(&tm[1], L->W_up, c.d, c.d_ff, c.d, 128) &&
+           make_map(&tm[2], X ? X : plan->x_bf16, c.d, B, c.d, N) &&
+           make_map(&tm[3], X_lo ? X_lo : plan->x_bf16, c.d, B, c.d, N) &&
+           make_map(&tm[4], L->Wd_t, c.d, c.d_ff, c.d, BK) &&
+           make_map(&tm[5], actT, 128, (uint64_t)plan->G * 128, 128, BK) &&
+           make_map(&tm[6], actT_lo, 128, (uint64_t)plan->G * 128, 128, BK);
+}
+
+cs_status launch_decode_gateup(cs_plan *plan, const cs_layer *L, const void *X, const void *X_lo, int B,
+                               bool masked, cudaStream_t st) {
     const cs_config &c = plan->cfg;
     const int N = (B + 15) / 16 * 16;
     __nv_bfloat16 *actT = static_cast<__nv_bfloat16 *>(plan->act);
     __nv_bfloat16 *actT_lo = actT + (size_t)plan->G * 128 * 128;
-    CUtensorMap tm_g, tm_u, tm_x, tm_x_lo, tm_wd, tm_act, tm_act_lo;
-    if (!make_map(&tm_g, L->W_gate, c.d, c.d_ff, c.d, 128) || !make_map(&tm_u, L->W_up, c.d, c.d_ff, c.d, 128) ||
-        !make_map(&tm_x, X, c.d, B, c.d, N) || !make_map(&tm_x_lo, X_lo, c.d, B, c.d, N) ||
-        !make_map(&tm_wd, L->Wd_t, c.d, c.d_ff, c.d, BK) ||
-        !make_map(&tm_act, actT, 128, (uint64_t)plan->G * 128, 128, BK) ||
-        !make_map(&tm_act_lo, actT_lo, 128, (uint64_t)plan->G * 128, 128, BK))
-        return record_cuda(plan, cudaErrorInvalidValue, "cuTensorMapEncodeTiled");
+    CUtensorMap tm[7];
+    if (!decode_maps(plan, L, X, X_lo, B, N, tm)) return record_cuda(plan, cudaErrorInvalidValue, "cuTensorMapEncodeTiled");
+    StageTimer timer(plan, CS_STAGE_EXEC, st);
+    ffn_gateup_swap_kernel<true><<<plan->G, kMmaThreads, kMmaSmem, st>>>(
+        tm[0], tm[1], tm[2], tm[3], masked ? plan->glist : nullptr, plan->nu, N, c.d,
+        masked ? plan->gmask : nullptr, actT, actT_lo, plan->status);
+    plan->launches++;
+    CS_CUDA_TRY(plan, cudaGetLastError());
+    return CS_OK;
+}
+
+cs_status launch_decode_mask(cs_plan *plan, int B, cudaStream_t st) {
+    const int N = (B + 15) / 16 * 16;
+    __nv_bfloat16 *actT = static_cast<__nv_bfloat16 *>(plan->act);
+    __nv_bfloat16 *actT_lo = actT + (size_t)plan->G * 128 * 128;
+    const int rows = plan->G * 128, total = rows * (N / 8);
+    mask_act_kernel<<<(total + 255) / 256, 256, 0, st>>>(actT, actT_lo, plan->gmask, rows, N);
+    plan->launches++;
+    CS_CUDA_TRY(plan, cudaGetLastError());
+    return CS_OK;
+}
+
+cs_status launch_decode_down(cs_plan *plan, const cs_layer *L, int B, bool act_by_group, const float *residual,
+                             float *out, cudaStream_t st) {
+    const cs_config &c = plan->cfg;
+    const int N = (B + 15) / 16 * 16;
+    CUtensorMap tm[7];
+    if (!decode_maps(plan, L, nullptr, nullptr, B, N, tm)) return record_cuda(plan, cudaErrorInvalidValue, "cuTensorMapEncodeTiled");
     const int Z = max(1, min(plan->sm_count / (c.d / 128), 8));
     {
-        StageTimer timer(plan, CS_STAGE_EXEC, st);
-        ffn_gateup_swap_kernel<true><<<plan->G, kMmaThreads, kMmaSmem, st>>>(
-            tm_g, tm_u, tm_x, tm_x_lo, plan->glist, plan->nu, N, c.d, plan->gmask, actT, actT_lo, plan->status);
-        plan->launches++;
-        CS_CUDA_TRY(plan, cudaGetLastError());
+        StageTimer timer(plan, CS_STAGE_EXEC2, st);
         ffn_down_swap_kernel<true><<<dim3(c.d / 128, Z), kMmaThreads, kMmaSmem, st>>>(
-            tm_wd, tm_act, tm_act_lo, plan->glist, plan->nu, N, B, c.d, plan->mma_partial, plan->status);
+            tm[4], tm[5], tm[6], plan->glist, plan->nu, N, B, c.d, act_by_group ? 1 : 0, plan->mma_partial, plan->status);
         plan->launches++;
         CS_CUDA_TRY(plan, cudaGetLastError());
     }

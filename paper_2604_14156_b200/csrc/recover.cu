@@ -169,9 +169,9 @@ cs_status launch_recover(cs_plan *plan, const float *Phi, float mu, const float 
     const int warps = (G + 31) / 32;
     const size_t smem = sizeof(float) * ((size_t)c.m * (G | 1) + 4 * kMaxG + kRecMaxWarps * kMaxM + kRecMaxWarps);
     if (c.m <= 32)
-        launch_pdl(recover_kernel<1>, dim3(B), dim3(32 * warps), smem, st, Phi, mu, y, c.m, G, c.k, c.T, support, z, resid);
+        launch_pdl(pdl_for(plan, B), recover_kernel<1>, dim3(B), dim3(32 * warps), smem, st, Phi, mu, y, c.m, G, c.k, c.T, support, z, resid);
     else
-        launch_pdl(recover_kernel<2>, dim3(B), dim3(32 * warps), smem, st, Phi, mu, y, c.m, G, c.k, c.T, support, z, resid);
+        launch_pdl(pdl_for(plan, B), recover_kernel<2>, dim3(B), dim3(32 * warps), smem, st, Phi, mu, y, c.m, G, c.k, c.T, support, z, resid);
     plan->launches++;
     CS_CUDA_TRY(plan, cudaGetLastError());
     return CS_OK;

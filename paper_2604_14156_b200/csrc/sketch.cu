@@ -95,7 +95,7 @@ cs_status launch_sketch(cs_plan *plan, const float *S, const float *x, const flo
     dim3 grid((c.m + rpc - 1) / rpc, B);
     const int cpt = (c.d / 4 + kSketchThreads - 1) / kSketchThreads;
 #define CS_SKETCH_CASE(N)                                                                            \
-    launch_pdl(sketch_kernel<N>, grid, dim3(kSketchThreads), 0, st, S, x, gamma, c.rms_eps, c.m, c.d, rpc, y, n_out)
+    launch_pdl(pdl_for(plan, B), sketch_kernel<N>, grid, dim3(kSketchThreads), 0, st, S, x, gamma, c.rms_eps, c.m, c.d, rpc, y, n_out)
     if (cpt <= 1) CS_SKETCH_CASE(1);
     else if (cpt <= 2) CS_SKETCH_CASE(2);
     else if (cpt <= 4) CS_SKETCH_CASE(4);
