@@ -27,6 +27,7 @@ if ROOT not in sys.path:
 import torch  # noqa: E402
 
 from gen import workloads as W  # noqa: E402
+from paper_2604_14156_b200 import shard  # noqa: E402
 
 METRIC = "sparse_ffn_decode_tokens_per_s_per_layer"
 UNIT = "tokens/s"
@@ -152,7 +153,7 @@ def run_ours(args):
         layers_raw.append(L)
         layers.append(cs.Layer(plan, L.S, L.Phi, L.W_gate, L.W_up, L.Wd_t, L.mu, L.gamma, cfg.rms))
     # each rank decodes its own tokens (weak scaling): the batch index is offset by the rank
-    xs = torch.stack([W.make_tokens(cfg, layers_raw[0].A, batch=rank * N_TOKEN_BATCHES + j).h
+    xs = torch.stack([W.make_tokens(cfg, layers_raw[0].A, batch=shard.batch_stream(rank, j, N_TOKEN_BATCHES)).h
                       for j in range(N_TOKEN_BATCHES)]).to(dev)
     x_out = torch.empty_like(xs[0])
     sup_probe = None
