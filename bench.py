@@ -31,6 +31,13 @@ from paper_2604_14156_b200 import shard  # noqa: E402
 
 METRIC = "sparse_ffn_decode_tokens_per_s_per_layer"
 UNIT = "tokens/s"
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the roofline kernels, from the
+# ncu captures summarised under profiles/, keyed by (workload, k).  An entry is removed when its
+# kernel changes and comes back with the next capture; a missing entry reports null.
+NCU_TRAFFIC = {
+    ("l2_7b_b64", 22): 185.52e6 + 99.51e6,      # ffn_gateup_swap_kernel + ffn_down_swap_kernel
+    ("l2_13b_prompt", 27): 216.33e6 + 77.39e6,  # ffn_gateup_mma_kernel + ffn_down_mma_kernel
+}
 GRAPH_STEPS = 64          # steps captured per CUDA graph
 N_TOKEN_BATCHES = 16      # distinct input batches rotated through
 
@@ -275,11 +282,13 @@ def run_ours(args):
         "gpu_launches": int(round(launches_per_step * K)),
         "clocks": clocks.summary(),
         "roofline": {"bound": "hbm",
-                     "kernel": "ffn_gateup_mma_kernel + ffn_down_mma_kernel" if mma else "ffn_gather_kernel",
+                     "kernel": ("ffn_gateup_swap_kernel + ffn_down_swap_kernel" if cfg.B <= 128 else
+                                "ffn_gateup_mma_kernel + ffn_down_mma_kernel") if mma else "ffn_gather_kernel",
                      "achieved": achieved, "peak": peak,
                      "unit": "GB/s", "frac": (achieved / peak) if achieved else None, "peak_kind": peak_kind,
                      "frac_of_8tbs_nominal": (achieved / 8000.0) if achieved else None,
-                     "bytes_per_launch": kernel_bytes, "avg_launch_us": exec_ms * 1e3, "traffic": None},
+                     "bytes_per_launch": kernel_bytes, "avg_launch_us": exec_ms * 1e3,
+                     "traffic": NCU_TRAFFIC.get((cfg.name, cfg.k))},
         "stages_us": {"sketch": stage_ms[0] * 1e3, "recover": stage_ms[1] * 1e3, "exec": stage_ms[2] * 1e3,
                       "exec_down": stage_ms[4] * 1e3, "reduce": stage_ms[3] * 1e3, "step_net": step_us,
                       "measure_recover_per_token": mr_us / cfg.B,
@@ -389,7 +398,8 @@ def run_prompt(args, cfg, rank, world, local, dev):
         "gpu_launches": launches, "clocks": clocks.summary(),
         "roofline": {"bound": "tensor", "kernel": "ffn_gateup_mma_kernel + ffn_down_mma_kernel", "achieved": achieved,
                      "peak": tf_peak, "unit": "TFLOP/s", "frac": achieved / tf_peak, "peak_kind": kind + " (sustained)",
-                     "flops_per_launch_pair": flops, "avg_pair_us": stage_ms[2] * 1e3, "traffic": None},
+                     "flops_per_launch_pair": flops, "avg_pair_us": stage_ms[2] * 1e3,
+                     "traffic": NCU_TRAFFIC.get((cfg.name, cfg.k))},
         "stages_us": {"mean_sketch": stage_ms[0] * 1e3, "recover": stage_ms[1] * 1e3, "exec": stage_ms[2] * 1e3,
                       "reduce": stage_ms[3] * 1e3, "step_net": ms_total * 1e3 / K},
     }
