@@ -59,6 +59,7 @@ cs_status cs_plan_create(const cs_config *cfg, cs_plan **out) {
     alloc((void **)&p->z_buf, nt * cfg->k * sizeof(float));
     alloc((void **)&p->resid_buf, nt * sizeof(float));
     alloc((void **)&p->partial, (size_t)kGatherMaxTokens * p->nx_max * cfg->d * sizeof(float));
+    alloc((void **)&p->gram, (size_t)kMaxG * kMaxG * sizeof(float));
     alloc((void **)&p->hbar, (size_t)cfg->d * sizeof(float));
     alloc((void **)&p->colsum, (size_t)p->mean_row_blocks * cfg->d * sizeof(float));
     alloc((void **)&p->status, sizeof(DeviceStatus));
@@ -87,6 +88,7 @@ cs_status cs_plan_create(const cs_config *cfg, cs_plan **out) {
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p->ev_fork, cudaEventDisableTiming);
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p->ev_join, cudaEventDisableTiming);
     if (e == cudaSuccess) e = cudaMemset(p->status, 0, sizeof(DeviceStatus));
+    if (e == cudaSuccess && prepare_recover(p) != CS_OK) e = cudaErrorUnknown;
     if (e == cudaSuccess && prepare_ffn_gather(p) != CS_OK) e = cudaErrorUnknown;
     if (e == cudaSuccess && p->mma_ok && prepare_ffn_mma(p) != CS_OK) e = cudaErrorUnknown;
     if (e != cudaSuccess) {
@@ -100,7 +102,7 @@ cs_status cs_plan_create(const cs_config *cfg, cs_plan **out) {
 cs_status cs_plan_destroy(cs_plan *p) {
     if (p == nullptr) return CS_ERR_NULL;
     cudaFree(p->n_buf); cudaFree(p->y_buf); cudaFree(p->sup_buf); cudaFree(p->z_buf);
-    cudaFree(p->resid_buf); cudaFree(p->partial); cudaFree(p->hbar); cudaFree(p->colsum);
+    cudaFree(p->resid_buf); cudaFree(p->partial); cudaFree(p->gram); cudaFree(p->hbar); cudaFree(p->colsum);
     cudaFree(p->status); cudaFree(p->x_host_in); cudaFree(p->x_host_out);
     cudaFree(p->mask); cudaFree(p->gmask); cudaFree(p->counts); cudaFree(p->offsets); cudaFree(p->token_ids); cudaFree(p->glist);
     cudaFree(p->nu); cudaFree(p->x_bf16); cudaFree(p->act); cudaFree(p->mma_partial);
@@ -117,7 +119,7 @@ cs_status cs_sketch(cs_plan *plan, const float *S, const float *h, int32_t B, fl
     if (plan == nullptr || S == nullptr || h == nullptr || y == nullptr) return CS_ERR_NULL;
     if (B <= 0 || B > plan->cfg.max_tokens) return CS_ERR_SHAPE;
     if (!aligned16(S) || !aligned16(h)) return CS_ERR_UNSUPPORTED;
-    return launch_sketch(plan, S, h, nullptr, B, y, nullptr, static_cast<cudaStream_t>(stream));
+    return launch_sketch(plan, S, h, nullptr, B, y, nullptr, nullptr, 0.f, static_cast<cudaStream_t>(stream));
 }
 
 cs_status cs_recover(cs_plan *plan, const float *Phi, float mu, const float *y, int32_t B,
@@ -125,7 +127,7 @@ cs_status cs_recover(cs_plan *plan, const float *Phi, float mu, const float *y, 
     if (plan == nullptr || Phi == nullptr || y == nullptr || support == nullptr) return CS_ERR_NULL;
     if (B <= 0 || B > plan->cfg.max_tokens) return CS_ERR_SHAPE;
     if (!isfinite(mu) || !(mu > 0.f)) return CS_ERR_NONFINITE;
-    return launch_recover(plan, Phi, mu, y, B, support, z, resid, static_cast<cudaStream_t>(stream));
+    return launch_recover(plan, Phi, mu, y, B, support, z, resid, false, static_cast<cudaStream_t>(stream));
 }
 
 static cs_status check_weights(const cs_layer *L) {
@@ -223,21 +225,21 @@ cs_status cs_layer_step(cs_plan *plan, const cs_layer *layer, const float *x, in
     if (use_decode_mma(plan, B)) {
         // recovery (and, without a normalisation to wait for, the sketch too) beside the gate/up GEMM
         if (norm) {
-            s = launch_sketch(plan, layer->S, x, layer->rms_gamma, B, plan->y_buf, plan->n_buf, st);
+            s = launch_sketch(plan, layer->S, x, layer->rms_gamma, B, plan->y_buf, plan->n_buf, layer->Phi, layer->mu, st);
             if (s != CS_OK) return s;
         }
         return exec_decode_overlapped(plan, layer, n, B, layer->add_residual ? x : nullptr, x_out, st,
                                       [&](cudaStream_t side) {
             cs_status r = CS_OK;
-            if (!norm) r = launch_sketch(plan, layer->S, x, nullptr, B, plan->y_buf, nullptr, side);
-            if (r == CS_OK) r = launch_recover(plan, layer->Phi, layer->mu, plan->y_buf, B, sup, z_out, resid_out, side);
+            if (!norm) r = launch_sketch(plan, layer->S, x, nullptr, B, plan->y_buf, nullptr, layer->Phi, layer->mu, side);
+            if (r == CS_OK) r = launch_recover(plan, layer->Phi, layer->mu, plan->y_buf, B, sup, z_out, resid_out, true, side);
             if (r == CS_OK) r = launch_bucket(plan, sup, B, side);
             return r;
         });
     }
-    s = launch_sketch(plan, layer->S, x, layer->rms_gamma, B, plan->y_buf, norm ? plan->n_buf : nullptr, st);
+    s = launch_sketch(plan, layer->S, x, layer->rms_gamma, B, plan->y_buf, norm ? plan->n_buf : nullptr, layer->Phi, layer->mu, st);
     if (s != CS_OK) return s;
-    s = launch_recover(plan, layer->Phi, layer->mu, plan->y_buf, B, sup, z_out, resid_out, st);
+    s = launch_recover(plan, layer->Phi, layer->mu, plan->y_buf, B, sup, z_out, resid_out, true, st);
     if (s != CS_OK) return s;
     // supports produced by cs_recover are valid by construction: no device check here
     return exec_dispatch(plan, layer, n, sup, B, layer->add_residual ? x : nullptr, x_out, st);
@@ -290,9 +292,9 @@ cs_status cs_prompt_support(cs_plan *plan, const float *S, const float *Phi, flo
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     cs_status s = launch_prompt_mean(plan, H, n, plan->hbar, st);
     if (s != CS_OK) return s;
-    s = launch_sketch(plan, S, plan->hbar, nullptr, 1, plan->y_buf, nullptr, st);
+    s = launch_sketch(plan, S, plan->hbar, nullptr, 1, plan->y_buf, nullptr, Phi, mu, st);
     if (s != CS_OK) return s;
-    return launch_recover(plan, Phi, mu, plan->y_buf, 1, support, z, resid, st);
+    return launch_recover(plan, Phi, mu, plan->y_buf, 1, support, z, resid, true, st);
 }
 
 cs_status cs_ffn_exec_shared(cs_plan *plan, const cs_layer *layer, const void *H, int32_t n,

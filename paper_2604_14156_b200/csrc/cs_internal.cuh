@@ -37,6 +37,7 @@ struct cs_plan {
     float *z_buf;      // [max_tokens, k]
     float *resid_buf;  // [max_tokens]
     float *partial;    // [kGatherMaxTokens, nx_max, d] partial down-projections of the gather path
+    float *gram;       // [G, pitch] I - mu Phi^T Phi of the layer being recovered, pitch = 32 ceil(G/32)
     float *hbar;       // [d] mean prompt hidden state
     float *colsum;     // [mean_row_blocks, d]
     cs::DeviceStatus *status;  // device status word
@@ -89,10 +90,13 @@ struct StageTimer {
 };
 
 // Kernel launchers (each enqueues on `st`, bumps plan->launches, returns a status).
+// Phi != NULL: the launch also forms the recovery's matrix I - mu Phi^T Phi (plan->gram) in spare CTAs.
 cs_status launch_sketch(cs_plan *plan, const float *S, const float *x, const float *gamma, int B,
-                        float *y, float *n_out, cudaStream_t st);
+                        float *y, float *n_out, const float *Phi, float mu, cudaStream_t st);
+// gram_ready: plan->gram already holds this Phi's matrix (the sketch launch before formed it).
 cs_status launch_recover(cs_plan *plan, const float *Phi, float mu, const float *y, int B,
-                         int32_t *support, float *z, float *resid, cudaStream_t st);
+                         int32_t *support, float *z, float *resid, bool gram_ready, cudaStream_t st);
+cs_status prepare_recover(cs_plan *plan);
 cs_status launch_ffn_gather(cs_plan *plan, const cs_layer *layer, const float *h, const int32_t *support,
                             int B, const float *residual, float *out, cudaStream_t st);
 cs_status prepare_ffn_gather(cs_plan *plan);
@@ -135,6 +139,32 @@ inline cudaError_t launch_pdl(bool pdl, void (*kernel)(KArgs...), dim3 grid, dim
 }
 
 // ---- small device helpers -------------------------------------------------------------------
+// Rows 2*blk and 2*blk+1 of M = I - mu Phi^T Phi by a CTA of kGramThreads threads.  M is stored
+// row-major with a pitch of 32 * ceil(G / 32) floats, the columns past G zero, so that a recovery
+// thread can read its row with aligned 16-byte loads and needs no bounds in its inner loop.
+// The values depend on parameters only and are computed at once; the store waits for the kernels
+// before this one, which may still be reading the previous layer's matrix.
+constexpr int kGramThreads = 256;
+inline int gram_blocks(int G) { return (G + 1) / 2; }
+__host__ __device__ inline int gram_pitch(int G) { return (G + 31) & ~31; }
+__device__ __forceinline__ void gram_rows(const float *__restrict__ Phi, float mu, int m, int G, int blk,
+                                          float *__restrict__ gram) {
+    const int a = blk * 2 + (threadIdx.x >> 7), b = threadIdx.x & 127;
+    const int pitch = gram_pitch(G);
+    const bool valid = a < G && b < G;
+    float s0 = 0.f, s1 = 0.f;
+    if (valid) {
+        int i = 0;
+        for (; i + 1 < m; i += 2) {
+            s0 = fmaf(__ldg(Phi + i * G + a), __ldg(Phi + i * G + b), s0);
+            s1 = fmaf(__ldg(Phi + (i + 1) * G + a), __ldg(Phi + (i + 1) * G + b), s1);
+        }
+        if (i < m) s0 = fmaf(__ldg(Phi + i * G + a), __ldg(Phi + i * G + b), s0);
+    }
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (a < G && b < pitch) gram[a * pitch + b] = valid ? (a == b ? 1.f : 0.f) - mu * (s0 + s1) : 0.f;
+}
+
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);

@@ -1,177 +1,268 @@
 // Estimator: block iterative hard thresholding, one small CTA per token.
 //
-//   z_0 = 0;  T times:  r = y - Phi z;  v = z + mu Phi^T r;  z = H_k(v)
+//   z_0 = 0;  T times:  v = z + mu Phi^T (y - Phi z);  z = H_k(v)
 //
-// The iteration is a latency chain (T sequential steps of two tiny mat-vecs and a top-k) whose
-// cost is the number of instructions on the critical path, so the CTA is as small as the data
-// allows: warp w owns entries 32w .. 32w+31 of v and z (one entry per lane, ceil(G/32) warps).
-//   - Phi (m x G) sits in shared memory with an odd row pitch (both access patterns conflict-free).
-//   - z is carried as a compact list of exactly k (index, value) pairs in shared memory.  Every
-//     warp rebuilds the residual r from that list on its own (lane i owns rows i and i+32), so no
-//     block barrier separates the two mat-vecs.
-//   - H_k is exact under the total order (|v| descending, group index ascending).  Keys are the
-//     float bit patterns of |v| (monotone for non-negative floats).  An entry's rank is the number
-//     of entries that precede it: key greater, or equal from a lower index.  Blocks of 32 keys
-//     owned by lower warps count with >=, by higher warps with >, and inside the own warp
-//     equal keys are found with one match instruction.  rank < k  <=>  kept, and the rank is the
-//     entry's slot in the new list, so the loop needs no prefix sum.
-// Two block barriers per iteration: keys visible, list visible.  After the last iteration the
-// kept entries are written in ascending index order, which is the output format.
+// The iteration is a latency chain (T sequential steps of a small mat-vec and a top-k), so the cost
+// is the number of instructions on the critical path.  Two things keep it short.
+//   - The update is evaluated in its expanded form  v = c + M z  with  c = mu Phi^T y  (once per
+//     token) and  M = I - mu Phi^T Phi  (once per layer, gram_rows below).  Since z has exactly k
+//     non-zeros, one iteration is k multiply-adds per entry instead of the two mat-vecs through
+//     the m-dimensional residual, and nothing but z crosses threads.
+//   - Thread g owns entry g of v and z (one entry per lane, ceil(G/32) warps).  z is a compact list
+//     of its k values in shared memory, read by broadcast, and the thread keeps the k matrix entries
+//     M[g, idx_j] that go with the list in registers, so the mat-vec has no indexed load.  (For
+//     k > 56 z is a dense vector instead and the thread keeps its whole row of M.)
+//   - H_k is exact under the total order (|v| descending, group index ascending), but most
+//     iterations do not change the support, which is the case exactly when every kept |v| exceeds
+//     every other |v|: two warp reductions and one barrier decide that, and only otherwise are the
+//     exact ranks computed.  A rank is the number of entries that precede: key greater, or equal
+//     from a lower index.  Blocks of 32 keys owned by lower warps count with >=, by higher warps
+//     with >.  Equal keys inside the own warp are rare (exact ties); they make the ranks add up to
+//     less than those of a permutation, which every thread checks, and only then is the slow match
+//     instruction used to put the lower index first.  rank < k  <=>  kept, and the rank is the
+//     entry's slot in the new list.
+// A shared-memory round trip costs about 30 cycles and a barrier about 20, so an iteration that
+// keeps the support is one round trip, one barrier and k multiply-adds.  After the last iteration
+// the kept entries are written in ascending index order (the output format) and ||y - Phi z||_2 is
+// formed from Phi, y and z.
 #include "cs_internal.cuh"
 
 namespace cs {
 
-constexpr int kRecMaxWarps = kMaxG / 32;
 
-template <int ROWS>  // residual rows per lane: ceil(m / 32)
-__global__ void __launch_bounds__(32 * kRecMaxWarps)
-recover_kernel(const float *__restrict__ Phi, float mu, const float *__restrict__ y, int m, int G, int k,
-               int T, int32_t *__restrict__ support, float *__restrict__ z_out, float *__restrict__ resid_out) {
-    extern __shared__ __align__(16) float smem[];
+// M = I - mu Phi^T Phi, row-major [G, G]; only Phi and mu enter, so it can be formed beside the sketch.
+__global__ void __launch_bounds__(kGramThreads) gram_kernel(const float *__restrict__ Phi, float mu, int m, int G,
+                                                            float *__restrict__ gram) {
+    pdl_launch_dependents();
+    gram_rows(Phi, mu, m, G, blockIdx.x, gram);
+}
+
+// 1.0f if a > b else 0.0f.
+__device__ __forceinline__ float gt01(float a, float b) {
+    float r;
+    asm("set.gt.f32.f32 %0, %1, %2;" : "=f"(r) : "f"(a), "f"(b));
+    return r;
+}
+__device__ __forceinline__ void cp_async16_rec(void *smem_dst, const void *gmem_src) {
+    const uint32_t s = static_cast<uint32_t>(__cvta_generic_to_shared(smem_dst));
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 16;" ::"r"(s), "l"(gmem_src) : "memory");
+}
+
+// NW = warps = ceil(G / 32).  KC = ceil(k / 8) for k <= 56: the iterate is a compact list of k
+// values whose matrix entries M[idx_j, g] the thread keeps in registers; KC = 0: any k, the iterate
+// is a dense vector and the thread keeps its whole row of M.
+template <int NW, int KC>
+__global__ void __launch_bounds__(32 * NW)
+recover_kernel(const float *__restrict__ Phi, const float *__restrict__ gram, float mu, const float *__restrict__ y,
+               int m, int G, int k, int T, int32_t *__restrict__ support, float *__restrict__ z_out,
+               float *__restrict__ resid_out) {
+    constexpr int GP = 32 * NW;                    // padded number of entries = pitch of M
+    constexpr int NV = KC > 0 ? KC * 8 : GP;       // length of the iterate as the mat-vec reads it
+    constexpr int NR = KC > 0 ? KC * 8 : GP;       // matrix entries a thread keeps
+    extern __shared__ __align__(16) float m_s[];   // [G][GP] (list form only)
+    __shared__ __align__(16) float key_s[GP];      // |v| of the current iterate
+    __shared__ __align__(16) float val_s[2][NV];   // the iterate, by iteration parity: list values, or dense z
+    __shared__ int idx_s[NV];                      // list form: entry index of each list slot
+    __shared__ float y_s[kMaxM];
+    __shared__ uint32_t mm_s[2][2][4];             // per parity: min kept key / max other key, per warp
+    __shared__ int sum_s[4];                       // rank sums per warp
+    __shared__ int cnt_s[4];
+    __shared__ float red_s[kMaxM];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int nwarps = blockDim.x >> 5;
     const int g = tid;  // entry owned by this thread
-    const int Gp = G | 1;
-    int *key_s = reinterpret_cast<int *>(smem);                          // [kMaxG] keys of the current v
-    float2 *list_s = reinterpret_cast<float2 *>(smem + kMaxG);           // [kMaxG] (index bits, value), 16-byte aligned
-    float *r_w = smem + 3 * kMaxG + warp * kMaxM;                        // [warps][kMaxM] residual
-    int *cnt_s = reinterpret_cast<int *>(smem + 3 * kMaxG + kRecMaxWarps * kMaxM);  // [kRecMaxWarps]
-    int *slot_s = cnt_s + kRecMaxWarps;                                             // [kMaxG] rank claims
-    float *phi_s = smem + 4 * kMaxG + kRecMaxWarps * kMaxM + kRecMaxWarps;          // [m][Gp]
-
+    const bool valid = g < G;
     const int t = blockIdx.x;
     pdl_launch_dependents();
-    for (int col = tid; col < G; col += blockDim.x) {
-#pragma unroll 8
-        for (int row = 0; row < m; ++row) phi_s[row * Gp + col] = __ldg(Phi + row * G + col);
-    }
-    pdl_wait();   // Phi is a parameter and was staged above; y comes from the sketch kernel
-    float yv[ROWS];
+    pdl_wait();   // y and M come from the kernel before
+    float mreg[NR];
+    if constexpr (KC > 0) {
+        for (int i = tid; i < G * (GP / 4); i += GP) cp_async16_rec(m_s + 4 * i, gram + 4 * i);
+        asm volatile("cp.async.commit_group;" ::: "memory");
+    } else {   // row g of M (M is symmetric: row g is the column that multiplies into entry g)
+        const float4 *src = reinterpret_cast<const float4 *>(gram + (size_t)(valid ? g : 0) * GP);
 #pragma unroll
-    for (int q = 0; q < ROWS; ++q) {
-        const int row = lane + 32 * q;
-        yv[q] = row < m ? y[(size_t)t * m + row] : 0.f;
-    }
-    // z_0 = 0 with the support the order assigns to an all-zero vector: indices 0..k-1.
-    // The list is padded to a multiple of 8 with (index 0, value 0) so that loops over it need no tail.
-    const int k8 = (k + 7) & ~7;
-    if (tid < k8) list_s[tid] = make_float2(__int_as_float(tid < k ? tid : 0), 0.f);
-    if (tid + blockDim.x < k8) list_s[tid + blockDim.x] = make_float2(__int_as_float(0), 0.f);
-    float zv = 0.f;
-    bool kept = g < k;
-    const unsigned lt_mask = (1u << lane) - 1u;
-    __syncthreads();
-
-    // r = y - Phi z from the list (four accumulators shorten the dependency chain); returns the
-    // residual of this lane's rows and leaves it in r_w for the whole warp
-    auto residual = [&](float (&rr)[ROWS]) {
-#pragma unroll
-        for (int q = 0; q < ROWS; ++q) {
-            const int row = min(lane + 32 * q, m - 1);
-            const float *prow = phi_s + row * Gp;
-            float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
-            for (int c = 0; c < k8; c += 8) {
-                // eight list entries at a time: all list loads, then all Phi loads, then the FMAs
-                const float4 *lq = reinterpret_cast<const float4 *>(list_s + c);
-                const float4 e01 = lq[0], e23 = lq[1], e45 = lq[2], e67 = lq[3];
-                const float p0 = prow[__float_as_int(e01.x)], p1 = prow[__float_as_int(e01.z)];
-                const float p2 = prow[__float_as_int(e23.x)], p3 = prow[__float_as_int(e23.z)];
-                const float p4 = prow[__float_as_int(e45.x)], p5 = prow[__float_as_int(e45.z)];
-                const float p6 = prow[__float_as_int(e67.x)], p7 = prow[__float_as_int(e67.z)];
-                a0 = fmaf(p0, e01.y, a0); a1 = fmaf(p1, e01.w, a1);
-                a2 = fmaf(p2, e23.y, a2); a3 = fmaf(p3, e23.w, a3);
-                a0 = fmaf(p4, e45.y, a0); a1 = fmaf(p5, e45.w, a1);
-                a2 = fmaf(p6, e67.y, a2); a3 = fmaf(p7, e67.w, a3);
-            }
-            rr[q] = yv[q] - ((a0 + a1) + (a2 + a3));
-            if (lane + 32 * q < m) r_w[lane + 32 * q] = rr[q];
+        for (int j = 0; j < GP / 4; ++j) {
+            const float4 q = __ldg(src + j);
+            mreg[4 * j] = q.x; mreg[4 * j + 1] = q.y; mreg[4 * j + 2] = q.z; mreg[4 * j + 3] = q.w;
         }
-    };
+    }
+    for (int row = tid; row < m; row += GP) y_s[row] = y[(size_t)t * m + row];
+    // z_0 = 0 with the support the order assigns to an all-zero vector: indices 0..k-1
+    for (int i = tid; i < NV; i += GP) {
+        val_s[0][i] = 0.f; val_s[1][i] = 0.f;
+        idx_s[i] = i < k ? i : 0;
+    }
+    bool kept = g < k;
+    int slot = g;
+    float v = 0.f;
+    __syncthreads();
+    // c_g = mu sum_i Phi[i,g] y_i
+    float cg = 0.f;
+    if (valid) {
+        float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+        const float *pcol = Phi + g;
+        int row = 0;
+#pragma unroll 4
+        for (; row + 3 < m; row += 4) {
+            a0 = fmaf(__ldg(pcol + row * G), y_s[row], a0); a1 = fmaf(__ldg(pcol + (row + 1) * G), y_s[row + 1], a1);
+            a2 = fmaf(__ldg(pcol + (row + 2) * G), y_s[row + 2], a2); a3 = fmaf(__ldg(pcol + (row + 3) * G), y_s[row + 3], a3);
+        }
+        for (; row < m; ++row) a0 = fmaf(__ldg(pcol + row * G), y_s[row], a0);
+        cg = mu * ((a0 + a1) + (a2 + a3));
+    }
+    const float *mcol = m_s + (valid ? g : 0);
+    if constexpr (KC > 0) {
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
+        __syncthreads();
+#pragma unroll
+        for (int j = 0; j < NR; ++j) mreg[j] = mcol[idx_s[j] * GP];
+    }
+    const unsigned lt_mask = (1u << lane) - 1u;
+    const int rank_total = G * (G - 1) / 2;   // what the ranks of G distinct positions add up to
 
     for (int it = 0; it < T; ++it) {
-        float rr[ROWS];
-        residual(rr);
-        __syncwarp();
-        // v_g = z_g + mu sum_i Phi[i,g] r_i
-        float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
-        if (g < G) {
-            const float *pcol = phi_s + g;
-            int row = 0;
-            for (; row + 7 < m; row += 8) {
-                const float4 r4 = *reinterpret_cast<const float4 *>(r_w + row);
-                const float4 r8 = *reinterpret_cast<const float4 *>(r_w + row + 4);
-                const float q0 = pcol[row * Gp], q1 = pcol[(row + 1) * Gp], q2 = pcol[(row + 2) * Gp],
-                            q3 = pcol[(row + 3) * Gp], q4 = pcol[(row + 4) * Gp], q5 = pcol[(row + 5) * Gp],
-                            q6 = pcol[(row + 6) * Gp], q7 = pcol[(row + 7) * Gp];
-                a0 = fmaf(q0, r4.x, a0); a1 = fmaf(q1, r4.y, a1); a2 = fmaf(q2, r4.z, a2); a3 = fmaf(q3, r4.w, a3);
-                a0 = fmaf(q4, r8.x, a0); a1 = fmaf(q5, r8.y, a1); a2 = fmaf(q6, r8.z, a2); a3 = fmaf(q7, r8.w, a3);
-            }
-            for (; row < m; ++row) a0 = fmaf(pcol[row * Gp], r_w[row], a0);
+        const int par = it & 1;
+        // v_g = c_g + sum_j M[g, idx_j] z_j, the iterate read by broadcast
+        float a0 = cg, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+#pragma unroll
+        for (int j = 0; j < NV / 4; ++j) {
+            const float4 zq = reinterpret_cast<const float4 *>(val_s[par])[j];
+            a0 = fmaf(mreg[4 * j], zq.x, a0); a1 = fmaf(mreg[4 * j + 1], zq.y, a1);
+            a2 = fmaf(mreg[4 * j + 2], zq.z, a2); a3 = fmaf(mreg[4 * j + 3], zq.w, a3);
         }
-        const float v = fmaf(mu, (a0 + a1) + (a2 + a3), zv);
-        // invalid entries get key -1: they precede nothing and nothing needs their rank
-        const int key = g < G ? (int)(__float_as_uint(v) & 0x7fffffffu) : -1;
+        v = (a0 + a1) + (a2 + a3);
+        // Keys are |v| (entries past G get -2: they precede nothing).
+        const uint32_t kbits = __float_as_uint(v) & 0x7fffffffu;
+        const float key = valid ? __uint_as_float(kbits) : -2.f;
+        // Most iterations leave the support as it is.  That is the case exactly when every kept key is
+        // greater than every other key, which two warp reductions and one barrier decide; the next
+        // iterate is written on that assumption and rewritten below when it fails.
+        const uint32_t wmin = __reduce_min_sync(0xffffffffu, kept ? kbits : 0xffffffffu);
+        const uint32_t wmax = __reduce_max_sync(0xffffffffu, (valid && !kept) ? kbits : 0u);
         key_s[g] = key;
+        if constexpr (KC > 0) { if (kept) val_s[par ^ 1][slot] = v; }
+        else val_s[par ^ 1][g] = kept ? v : 0.f;
+        if (lane == 0) { mm_s[par][0][warp] = wmin; mm_s[par][1][warp] = wmax; }
         __syncthreads();
-        int c0 = 0, c1 = 0, c2 = 0, c3 = 0, c4 = 0, c5 = 0, c6 = 0, c7 = 0;  // independent counters
-        for (int blk = 0; blk < nwarps; ++blk) {
-            const int4 *kq = reinterpret_cast<const int4 *>(key_s + 32 * blk);
+        uint32_t gmin = 0xffffffffu, gmax = 0u;
+#pragma unroll
+        for (int w = 0; w < NW; ++w) { gmin = min(gmin, mm_s[par][0][w]); gmax = max(gmax, mm_s[par][1][w]); }
+        if (gmin > gmax) continue;
+
+        // The support may change: exact ranks.  "a >= key" is evaluated as "a > the next float below
+        // key" (-1 below zero), so that one kind of compare serves both cases.
+        const float key_lo = kbits == 0u ? -1.f : __uint_as_float(kbits - 1u);
+        float c0 = 0.f, c1 = 0.f, c2 = 0.f, c3 = 0.f, c4 = 0.f, c5 = 0.f, c6 = 0.f, c7 = 0.f;  // independent counters
+#pragma unroll
+        for (int blk = 0; blk < NW; ++blk) {
+            const float4 *kq = reinterpret_cast<const float4 *>(key_s + 32 * blk);
             // entries of lower warps precede on ties (>=), own and higher warps only when greater
-            const int thr = key - (blk < warp ? 1 : 0);
+            const float thr = blk < warp ? key_lo : key;
 #pragma unroll
             for (int jj = 0; jj < 8; jj += 2) {
-                const int4 ka = kq[jj], kb2 = kq[jj + 1];
-                c0 += ka.x > thr; c1 += ka.y > thr; c2 += ka.z > thr; c3 += ka.w > thr;
-                c4 += kb2.x > thr; c5 += kb2.y > thr; c6 += kb2.z > thr; c7 += kb2.w > thr;
+                const float4 ka = kq[jj], kb2 = kq[jj + 1];
+                c0 += gt01(ka.x, thr); c1 += gt01(ka.y, thr); c2 += gt01(ka.z, thr); c3 += gt01(ka.w, thr);
+                c4 += gt01(kb2.x, thr); c5 += gt01(kb2.y, thr); c6 += gt01(kb2.z, thr); c7 += gt01(kb2.w, thr);
             }
         }
-        int rank = ((c0 + c1) + (c2 + c3)) + ((c4 + c5) + (c6 + c7));
-        // Equal keys inside the own warp were not ordered above, so they share a rank.  That is
-        // rare (exact ties), and shows as two lanes claiming one slot of a scratch table; only then
-        // is the slower match instruction used to put the lower lane first.
-        if (g < G) slot_s[rank] = g;
-        __syncwarp();
-        const bool clash = g < G && slot_s[rank] != g;
-        if (__any_sync(0xffffffffu, clash)) rank += __popc(__match_any_sync(0xffffffffu, key) & lt_mask);
-        kept = g < G && rank < k;
-        zv = kept ? v : 0.f;
-        if (kept) list_s[rank] = make_float2(__int_as_float(g), v);
+        int rank = valid ? (int)(((c0 + c1) + (c2 + c3)) + ((c4 + c5) + (c6 + c7))) : 0;
+        // Equal keys inside the own warp were ordered by neither side, so they share a rank and the
+        // ranks no longer add up to those of a permutation; only then is the slow match instruction
+        // used to put the lower index first.
+        const int wsum = __reduce_add_sync(0xffffffffu, rank);
+        if (lane == 0) sum_s[warp] = wsum;
         __syncthreads();
+        int total = 0;
+#pragma unroll
+        for (int w = 0; w < NW; ++w) total += sum_s[w];
+        if (total != rank_total) rank += __popc(__match_any_sync(0xffffffffu, __float_as_uint(key)) & lt_mask);
+        kept = valid && rank < k;   // the rank is the entry's slot in the new list
+        slot = rank;
+        if constexpr (KC > 0) { if (kept) { idx_s[slot] = g; val_s[par ^ 1][slot] = v; } }
+        else val_s[par ^ 1][g] = kept ? v : 0.f;
+        __syncthreads();
+        if constexpr (KC > 0) {
+#pragma unroll
+            for (int j = 0; j < NR; ++j) mreg[j] = mcol[idx_s[j] * GP];
+        }
     }
 
-    // final residual norm (warp 0), from the list of the last iteration
-    if (warp == 0 && resid_out != nullptr) {
-        float rr[ROWS];
-        residual(rr);
-        float ss = 0.f;
+    // residual norm ||y - Phi z||_2: warp w takes rows w, w + NW, ...; lanes stride over the entries
+    if (resid_out != nullptr) {
+        __syncthreads();
+        key_s[g] = (kept && T > 0) ? v : 0.f;   // dense z
+        __syncthreads();
+        for (int row = warp; row < m; row += NW) {
+            float a = 0.f;
 #pragma unroll
-        for (int q = 0; q < ROWS; ++q) ss += (lane + 32 * q < m) ? rr[q] * rr[q] : 0.f;
-        ss = warp_sum(ss);
-        if (lane == 0) resid_out[t] = sqrtf(ss);
+            for (int j = 0; j < NW; ++j) {
+                const int col = lane + 32 * j;
+                if (col < G) a = fmaf(__ldg(Phi + row * G + col), key_s[col], a);
+            }
+            a = warp_sum(a);
+            if (lane == 0) { const float r = y_s[row] - a; red_s[row] = r * r; }
+        }
     }
     // ascending index order: a kept entry goes to slot (number of kept entries with a lower index)
     const unsigned kb = __ballot_sync(0xffffffffu, kept);
     if (lane == 0) cnt_s[warp] = __popc(kb);
     __syncthreads();
     if (kept) {
-        int slot = __popc(kb & lt_mask);
-        for (int w = 0; w < warp; ++w) slot += cnt_s[w];
-        support[(size_t)t * k + slot] = g;
-        if (z_out != nullptr) z_out[(size_t)t * k + slot] = zv;
+        int o = __popc(kb & lt_mask);
+        for (int w = 0; w < warp; ++w) o += cnt_s[w];
+        support[(size_t)t * k + o] = g;
+        if (z_out != nullptr) z_out[(size_t)t * k + o] = T > 0 ? v : 0.f;
+    }
+    if (resid_out != nullptr && tid == 0) {
+        float ss = 0.f;
+        for (int row = 0; row < m; ++row) ss += red_s[row];
+        resid_out[t] = sqrtf(ss);
     }
 }
 
-cs_status launch_recover(cs_plan *plan, const float *Phi, float mu, const float *y, int B,
-                         int32_t *support, float *z, float *resid, cudaStream_t st) {
+typedef void (*RecoverFn)(const float *, const float *, float, const float *, int, int, int, int, int32_t *, float *, float *);
+static int recover_kc(int k) { return k <= 56 ? (k + 7) / 8 : 0; }
+template <int NW> static RecoverFn recover_fn_kc(int k) {
+    switch (recover_kc(k)) {
+        case 1: return recover_kernel<NW, 1>;
+        case 2: return recover_kernel<NW, 2>;
+        case 3: return recover_kernel<NW, 3>;
+        case 4: return recover_kernel<NW, 4>;
+        case 5: return recover_kernel<NW, 5>;
+        case 6: return recover_kernel<NW, 6>;
+        case 7: return recover_kernel<NW, 7>;
+        default: return recover_kernel<NW, 0>;
+    }
+}
+static RecoverFn recover_fn(int G, int k) {
+    switch ((G + 31) / 32) {
+        case 1: return recover_fn_kc<1>(k);
+        case 2: return recover_fn_kc<2>(k);
+        case 3: return recover_fn_kc<3>(k);
+        default: return recover_fn_kc<4>(k);
+    }
+}
+// dynamic shared memory: M in the list form
+static size_t recover_smem(int G, int k) { return recover_kc(k) > 0 ? sizeof(float) * (size_t)G * gram_pitch(G) : 0; }
+
+cs_status prepare_recover(cs_plan *plan) {
+    CS_CUDA_TRY(plan, cudaFuncSetAttribute(recover_fn(plan->G, plan->cfg.k), cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                           (int)recover_smem(plan->G, plan->cfg.k)));
+    return CS_OK;
+}
+
+cs_status launch_recover(cs_plan *plan, const float *Phi, float mu, const float *y, int B, int32_t *support,
+                         float *z, float *resid, bool gram_ready, cudaStream_t st) {
     const cs_config &c = plan->cfg;
     const int G = plan->G;
     StageTimer timer(plan, CS_STAGE_RECOVER, st);
-    const int warps = (G + 31) / 32;
-    const size_t smem = sizeof(float) * ((size_t)c.m * (G | 1) + 4 * kMaxG + kRecMaxWarps * kMaxM + kRecMaxWarps);
-    if (c.m <= 32)
-        launch_pdl(pdl_for(plan, B), recover_kernel<1>, dim3(B), dim3(32 * warps), smem, st, Phi, mu, y, c.m, G, c.k, c.T, support, z, resid);
-    else
-        launch_pdl(pdl_for(plan, B), recover_kernel<2>, dim3(B), dim3(32 * warps), smem, st, Phi, mu, y, c.m, G, c.k, c.T, support, z, resid);
+    if (!gram_ready) {
+        launch_pdl(pdl_for(plan, B), gram_kernel, dim3(gram_blocks(G)), dim3(kGramThreads), 0, st, Phi, mu, c.m, G, plan->gram);
+        plan->launches++;
+        CS_CUDA_TRY(plan, cudaGetLastError());
+    }
+    launch_pdl(pdl_for(plan, B), recover_fn(G, c.k), dim3(B), dim3(gram_pitch(G)), recover_smem(G, c.k), st, Phi,
+               (const float *)plan->gram, mu, y, c.m, G, c.k, c.T, support, z, resid);
     plan->launches++;
     CS_CUDA_TRY(plan, cudaGetLastError());
     return CS_OK;

@@ -8,7 +8,8 @@
 // thread owns the float4 chunks tid, tid+256, ... of the row, keeps the matching x chunks in
 // registers, and the per-row partial sums are folded by warp shuffles and one shared-memory hop.
 // With one token the grid is m CTAs of one row each, so the m*d*4 bytes of S are pulled by m SMs
-// at once; with a decode batch a CTA takes several rows per token.
+// at once; with a decode batch a CTA takes several rows per token.  When the recovery follows, a few
+// extra CTAs of the same launch form its matrix I - mu Phi^T Phi, which needs the parameters only.
 #include "cs_internal.cuh"
 
 namespace cs {
@@ -19,9 +20,15 @@ constexpr int kSketchMaxRows = 16;
 template <int CPT>
 __global__ void __launch_bounds__(kSketchThreads)
 sketch_kernel(const float *__restrict__ S, const float *__restrict__ x, const float *__restrict__ gamma,
-              float eps, int m, int d, int rows_per_cta, float *__restrict__ y, float *__restrict__ n_out) {
+              float eps, int m, int d, int rows_per_cta, float *__restrict__ y, float *__restrict__ n_out,
+              int sketch_blocks, const float *__restrict__ Phi, float mu, int G, float *__restrict__ gram) {
     __shared__ float red[kSketchMaxRows + 1][kSketchThreads / 32];
     __shared__ float total[kSketchMaxRows + 1];
+    if ((int)blockIdx.x >= sketch_blocks) {   // spare CTAs: the recovery's matrix for this layer
+        pdl_launch_dependents();
+        if (blockIdx.y == 0) gram_rows(Phi, mu, m, G, blockIdx.x - sketch_blocks, gram);
+        return;
+    }
     const int t = blockIdx.y;
     const int r0 = blockIdx.x * rows_per_cta;
     const int nrows = min(rows_per_cta, m - r0);
@@ -85,17 +92,20 @@ sketch_kernel(const float *__restrict__ S, const float *__restrict__ x, const fl
     }
 }
 
+static_assert(kGramThreads == kSketchThreads, "the spare CTAs of the sketch launch form the Gram rows");
+
 cs_status launch_sketch(cs_plan *plan, const float *S, const float *x, const float *gamma, int B,
-                        float *y, float *n_out, cudaStream_t st) {
+                        float *y, float *n_out, const float *Phi, float mu, cudaStream_t st) {
     const cs_config &c = plan->cfg;
     StageTimer timer(plan, CS_STAGE_SKETCH, st);
     // Enough CTAs to cover the SMs about twice, at most kSketchMaxRows rows per CTA.
     int rpc = (c.m * B + 2 * plan->sm_count - 1) / (2 * plan->sm_count);
     rpc = max(1, min(rpc, min(c.m, kSketchMaxRows)));
-    dim3 grid((c.m + rpc - 1) / rpc, B);
+    const int sblocks = (c.m + rpc - 1) / rpc;
+    dim3 grid(sblocks + (Phi != nullptr ? gram_blocks(plan->G) : 0), B);
     const int cpt = (c.d / 4 + kSketchThreads - 1) / kSketchThreads;
 #define CS_SKETCH_CASE(N)                                                                            \
-    launch_pdl(pdl_for(plan, B), sketch_kernel<N>, grid, dim3(kSketchThreads), 0, st, S, x, gamma, c.rms_eps, c.m, c.d, rpc, y, n_out)
+    launch_pdl(pdl_for(plan, B), sketch_kernel<N>, grid, dim3(kSketchThreads), 0, st, S, x, gamma, c.rms_eps, c.m, c.d, rpc, y, n_out, sblocks, Phi, mu, plan->G, plan->gram)
     if (cpt <= 1) CS_SKETCH_CASE(1);
     else if (cpt <= 2) CS_SKETCH_CASE(2);
     else if (cpt <= 4) CS_SKETCH_CASE(4);
