@@ -88,7 +88,6 @@ cs_status cs_plan_create(const cs_config *cfg, cs_plan **out) {
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p->ev_fork, cudaEventDisableTiming);
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p->ev_join, cudaEventDisableTiming);
     if (e == cudaSuccess) e = cudaMemset(p->status, 0, sizeof(DeviceStatus));
-    if (e == cudaSuccess && prepare_recover(p) != CS_OK) e = cudaErrorUnknown;
     if (e == cudaSuccess && prepare_ffn_gather(p) != CS_OK) e = cudaErrorUnknown;
     if (e == cudaSuccess && p->mma_ok && prepare_ffn_mma(p) != CS_OK) e = cudaErrorUnknown;
     if (e != cudaSuccess) {

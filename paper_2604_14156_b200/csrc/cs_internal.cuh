@@ -96,7 +96,6 @@ cs_status launch_sketch(cs_plan *plan, const float *S, const float *x, const flo
 // gram_ready: plan->gram already holds this Phi's matrix (the sketch launch before formed it).
 cs_status launch_recover(cs_plan *plan, const float *Phi, float mu, const float *y, int B,
                          int32_t *support, float *z, float *resid, bool gram_ready, cudaStream_t st);
-cs_status prepare_recover(cs_plan *plan);
 cs_status launch_ffn_gather(cs_plan *plan, const cs_layer *layer, const float *h, const int32_t *support,
                             int B, const float *residual, float *out, cudaStream_t st);
 cs_status prepare_ffn_gather(cs_plan *plan);

@@ -10,8 +10,9 @@
 //     the m-dimensional residual, and nothing but z crosses threads.
 //   - Thread g owns entry g of v and z (one entry per lane, ceil(G/32) warps).  z is a compact list
 //     of its k values in shared memory, read by broadcast, and the thread keeps the k matrix entries
-//     M[g, idx_j] that go with the list in registers, so the mat-vec has no indexed load.  (For
-//     k > 56 z is a dense vector instead and the thread keeps its whole row of M.)
+//     M[g, idx_j] that go with the list in registers (fetched from global memory when the support
+//     changes), so the mat-vec has no indexed load.  (For k > 56 z is a dense vector instead and
+//     the thread keeps its whole row of M.)
 //   - H_k is exact under the total order (|v| descending, group index ascending), but most
 //     iterations do not change the support, which is the case exactly when every kept |v| exceeds
 //     every other |v|: two warp reductions and one barrier decide that, and only otherwise are the
@@ -30,7 +31,7 @@
 namespace cs {
 
 
-// M = I - mu Phi^T Phi, row-major [G, G]; only Phi and mu enter, so it can be formed beside the sketch.
+// M = I - mu Phi^T Phi, row-major with padded rows; only Phi and mu enter, so it can be formed beside the sketch.
 __global__ void __launch_bounds__(kGramThreads) gram_kernel(const float *__restrict__ Phi, float mu, int m, int G,
                                                             float *__restrict__ gram) {
     pdl_launch_dependents();
@@ -43,11 +44,6 @@ __device__ __forceinline__ float gt01(float a, float b) {
     asm("set.gt.f32.f32 %0, %1, %2;" : "=f"(r) : "f"(a), "f"(b));
     return r;
 }
-__device__ __forceinline__ void cp_async16_rec(void *smem_dst, const void *gmem_src) {
-    const uint32_t s = static_cast<uint32_t>(__cvta_generic_to_shared(smem_dst));
-    asm volatile("cp.async.ca.shared.global [%0], [%1], 16;" ::"r"(s), "l"(gmem_src) : "memory");
-}
-
 // NW = warps = ceil(G / 32).  KC = ceil(k / 8) for k <= 56: the iterate is a compact list of k
 // values whose matrix entries M[idx_j, g] the thread keeps in registers; KC = 0: any k, the iterate
 // is a dense vector and the thread keeps its whole row of M.
@@ -59,7 +55,6 @@ recover_kernel(const float *__restrict__ Phi, const float *__restrict__ gram, fl
     constexpr int GP = 32 * NW;                    // padded number of entries = pitch of M
     constexpr int NV = KC > 0 ? KC * 8 : GP;       // length of the iterate as the mat-vec reads it
     constexpr int NR = KC > 0 ? KC * 8 : GP;       // matrix entries a thread keeps
-    extern __shared__ __align__(16) float m_s[];   // [G][GP] (list form only)
     __shared__ __align__(16) float key_s[GP];      // |v| of the current iterate
     __shared__ __align__(16) float val_s[2][NV];   // the iterate, by iteration parity: list values, or dense z
     __shared__ int idx_s[NV];                      // list form: entry index of each list slot
@@ -75,10 +70,7 @@ recover_kernel(const float *__restrict__ Phi, const float *__restrict__ gram, fl
     pdl_launch_dependents();
     pdl_wait();   // y and M come from the kernel before
     float mreg[NR];
-    if constexpr (KC > 0) {
-        for (int i = tid; i < G * (GP / 4); i += GP) cp_async16_rec(m_s + 4 * i, gram + 4 * i);
-        asm volatile("cp.async.commit_group;" ::: "memory");
-    } else {   // row g of M (M is symmetric: row g is the column that multiplies into entry g)
+    if constexpr (KC == 0) {   // row g of M (M is symmetric: row g is the column that multiplies into entry g)
         const float4 *src = reinterpret_cast<const float4 *>(gram + (size_t)(valid ? g : 0) * GP);
 #pragma unroll
         for (int j = 0; j < GP / 4; ++j) {
@@ -110,12 +102,13 @@ recover_kernel(const float *__restrict__ Phi, const float *__restrict__ gram, fl
         for (; row < m; ++row) a0 = fmaf(__ldg(pcol + row * G), y_s[row], a0);
         cg = mu * ((a0 + a1) + (a2 + a3));
     }
-    const float *mcol = m_s + (valid ? g : 0);
+    // List form: the entries M[idx_j, g] that go with the list come straight from global memory (M is
+    // 30 to 60 KB and stays in L1/L2) and are fetched again only when the support changes, which
+    // keeps the CTA's shared memory at 2 KB.
+    const float *mcol = gram + (valid ? g : 0);
     if constexpr (KC > 0) {
-        asm volatile("cp.async.wait_group 0;" ::: "memory");
-        __syncthreads();
 #pragma unroll
-        for (int j = 0; j < NR; ++j) mreg[j] = mcol[idx_s[j] * GP];
+        for (int j = 0; j < NR; ++j) mreg[j] = __ldg(mcol + idx_s[j] * GP);
     }
     const unsigned lt_mask = (1u << lane) - 1u;
     const int rank_total = G * (G - 1) / 2;   // what the ranks of G distinct positions add up to
@@ -183,7 +176,7 @@ recover_kernel(const float *__restrict__ Phi, const float *__restrict__ gram, fl
         __syncthreads();
         if constexpr (KC > 0) {
 #pragma unroll
-            for (int j = 0; j < NR; ++j) mreg[j] = mcol[idx_s[j] * GP];
+            for (int j = 0; j < NR; ++j) mreg[j] = __ldg(mcol + idx_s[j] * GP);
         }
     }
 
@@ -242,15 +235,6 @@ static RecoverFn recover_fn(int G, int k) {
         default: return recover_fn_kc<4>(k);
     }
 }
-// dynamic shared memory: M in the list form
-static size_t recover_smem(int G, int k) { return recover_kc(k) > 0 ? sizeof(float) * (size_t)G * gram_pitch(G) : 0; }
-
-cs_status prepare_recover(cs_plan *plan) {
-    CS_CUDA_TRY(plan, cudaFuncSetAttribute(recover_fn(plan->G, plan->cfg.k), cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                           (int)recover_smem(plan->G, plan->cfg.k)));
-    return CS_OK;
-}
-
 cs_status launch_recover(cs_plan *plan, const float *Phi, float mu, const float *y, int B, int32_t *support,
                          float *z, float *resid, bool gram_ready, cudaStream_t st) {
     const cs_config &c = plan->cfg;
@@ -261,7 +245,7 @@ cs_status launch_recover(cs_plan *plan, const float *Phi, float mu, const float 
         plan->launches++;
         CS_CUDA_TRY(plan, cudaGetLastError());
     }
-    launch_pdl(pdl_for(plan, B), recover_fn(G, c.k), dim3(B), dim3(gram_pitch(G)), recover_smem(G, c.k), st, Phi,
+    launch_pdl(pdl_for(plan, B), recover_fn(G, c.k), dim3(B), dim3(gram_pitch(G)), 0, st, Phi,
                (const float *)plan->gram, mu, y, c.m, G, c.k, c.T, support, z, resid);
     plan->launches++;
     CS_CUDA_TRY(plan, cudaGetLastError());

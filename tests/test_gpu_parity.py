@@ -82,6 +82,39 @@ def test_recover_edge_cases():
             assert np.array_equal(sup[t].cpu().numpy(), ref.support)
 
 
+@pytest.mark.parametrize("name,k", [("l2_7b_b64", 22), ("l3_8b_stack", 28), ("l3_8b_stack", 60)])
+def test_recover_ties_across_warps(name, k):
+    """Exact ties between groups owned by different warps and by the same warp (duplicated and
+    negated columns of Phi), for the list form (k <= 56) and the dense form (k = 60) of the kernel."""
+    cfg = W.CONFIGS[name].with_(k=k)
+    Phi = rng.normal(cfg.seed, (W.T_PHI, 3), (cfg.m, cfg.G), dtype=torch.float32, scale=cfg.m ** -0.5)
+    Phi[:, 70] = Phi[:, 3]; Phi[:, 40] = -Phi[:, 35]; Phi[:, 71] = Phi[:, 3]; Phi[:, 10] = Phi[:, 9]
+    mu = W.spectral_step(Phi)
+    B = 16
+    y = rng.normal(cfg.seed, (78,), (B, cfg.m), dtype=torch.float32)
+    y[0] = 0.0                                      # every comparison a tie
+    plan = make_plan(cfg, max_tokens=B)
+    sup, z, resid = cs.cs_recover(plan, Phi.to(DEV), mu, y.to(DEV))
+    sup = sup.cpu().numpy(); z = z.cpu().numpy()
+    assert sup[0].tolist() == list(range(k)) and not z[0].any()
+    checked = 0
+    for t in range(1, B):
+        ref = oracle.iht(Phi, y[t], cfg.k, cfg.T, mu)
+        if np.array_equal(sup[t], ref.support):
+            assert rel(z[t], ref.z[ref.support]) <= Z_TOL
+            checked += 1
+        else:
+            assert ref.min_gap <= GAP_TOL
+    assert checked >= B - 3
+    # one iteration only: v = mu Phi^T y has the exact ties, and they decide the support directly
+    plan1 = make_plan(cfg.with_(T=1), max_tokens=B)
+    sup1, _, _ = cs.cs_recover(plan1, Phi.to(DEV), mu, y.to(DEV))
+    for t in range(1, B):
+        one = oracle.iht(Phi, y[t], cfg.k, 1, mu)
+        if one.min_gap > GAP_TOL or one.min_gap == 0.0:
+            assert np.array_equal(sup1[t].cpu().numpy(), one.support), t
+
+
 @pytest.mark.parametrize("name,B", [("tiny_f32", 4), ("l2_7b_b1", 1), ("l2_7b_b64", 3)])
 def test_ffn_exec_matches_oracle_on_given_supports(name, B):
     cfg = W.CONFIGS[name]
