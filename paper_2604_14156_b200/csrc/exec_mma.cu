@@ -324,7 +324,8 @@ __global__ void __launch_bounds__(kMmaThreads, 1)
 ffn_down_mma_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant__ CUtensorMap tm_act_lo,
                     const __grid_constant__ CUtensorMap tm_wd, const int32_t *__restrict__ glist,
                     const int32_t *__restrict__ ng_dev, int ng_host, int M, int m_pad, int d,
-                    float *__restrict__ partial, DeviceStatus *status) {
+                    float *__restrict__ partial, const float *residual, float *out_f32,
+                    __nv_bfloat16 *__restrict__ out_bf16, DeviceStatus *status) {
     constexpr int kStages = Ring<SPLIT>::kStages;
     extern __shared__ uint8_t smem_raw[];
     const int nt = blockIdx.x, mt = blockIdx.y, z = blockIdx.z, Z = gridDim.z;
@@ -361,12 +362,42 @@ ffn_down_mma_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_con
         } else if (mbar_wait(&t.bars->acc_ready, 0, t.bars, status)) {
             tc_fence_after();
             const uint32_t tbase = t.bars->tmem_base + ((uint32_t)(q * 32) << 16);
+            const size_t o = (size_t)m * d + (size_t)nt * BN;      // one slice: the tile is the output itself
 #pragma unroll 1
             for (int c = 0; c < BN / 32; ++c) {
                 uint32_t v[32];
                 tc_ld32(tbase + c * 32, v);
                 tc_wait_ld();
-                if (m < M) {
+                if (Z == 1) {
+                    if (m < M) {
+                        if (residual != nullptr) {
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) {
+                                const float4 r = *reinterpret_cast<const float4 *>(residual + o + c * 32 + 4 * j);
+                                v[4 * j] = __float_as_uint(__uint_as_float(v[4 * j]) + r.x);
+                                v[4 * j + 1] = __float_as_uint(__uint_as_float(v[4 * j + 1]) + r.y);
+                                v[4 * j + 2] = __float_as_uint(__uint_as_float(v[4 * j + 2]) + r.z);
+                                v[4 * j + 3] = __float_as_uint(__uint_as_float(v[4 * j + 3]) + r.w);
+                            }
+                        }
+                        if (out_f32 != nullptr) {
+#pragma unroll
+                            for (int j = 0; j < 8; ++j)
+                                *reinterpret_cast<uint4 *>(out_f32 + o + c * 32 + 4 * j) = make_uint4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) {
+                                uint32_t pk[4];
+#pragma unroll
+                                for (int e = 0; e < 4; ++e) {
+                                    const __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(v[8 * j + 2 * e]), __uint_as_float(v[8 * j + 2 * e + 1]));
+                                    pk[e] = *reinterpret_cast<const uint32_t *>(&h2);
+                                }
+                                *reinterpret_cast<uint4 *>(out_bf16 + o + c * 32 + 8 * j) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                            }
+                        }
+                    }
+                } else if (m < M) {
 #pragma unroll
                     for (int j = 0; j < 8; ++j)
                         *reinterpret_cast<uint4 *>(dst + c * 32 + 4 * j) = make_uint4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
@@ -836,15 +867,17 @@ cs_status launch_ffn_mma(cs_plan *plan, const cs_layer *L, const void *X, const 
         if (mtiles * ntiles < plan->sm_count) Z = max(1, min(plan->sm_count / (mtiles * ntiles), plan->mma_slices));
         if (split)
             ffn_down_mma_kernel<true><<<dim3(ntiles, mtiles, Z), kMmaThreads, kMmaSmem, st>>>(
-                tm_act, tm_act_lo, tm_wd, glist, ng_dev, ng_host, M, m_pad, c.d, plan->mma_partial, plan->status);
+                tm_act, tm_act_lo, tm_wd, glist, ng_dev, ng_host, M, m_pad, c.d, plan->mma_partial, residual, out_f32,
+                static_cast<__nv_bfloat16 *>(out_bf16), plan->status);
         else
             ffn_down_mma_kernel<false><<<dim3(ntiles, mtiles, Z), kMmaThreads, kMmaSmem, st>>>(
-                tm_act, tm_act_lo, tm_wd, glist, ng_dev, ng_host, M, m_pad, c.d, plan->mma_partial, plan->status);
+                tm_act, tm_act_lo, tm_wd, glist, ng_dev, ng_host, M, m_pad, c.d, plan->mma_partial, residual, out_f32,
+                static_cast<__nv_bfloat16 *>(out_bf16), plan->status);
         plan->launches++;
         CS_CUDA_TRY(plan, cudaGetLastError());
         plan->last_slices = Z;
     }
-    {
+    if (plan->last_slices > 1) {   // a single slice has written the output itself
         StageTimer timer(plan, CS_STAGE_REDUCE, st);
         const size_t total4 = (size_t)M * c.d / 4;
         const int blocks = (int)((total4 + 255) / 256);
