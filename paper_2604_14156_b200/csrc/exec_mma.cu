@@ -534,15 +534,18 @@ ffn_gateup_swap_kernel(const __grid_constant__ CUtensorMap tm_g, const __grid_co
     teardown_cta(bars, warp, tcols);
 }
 
-// grid (d / 128 output-column tiles, slices).  partial [slice][128 tokens][d].
-template <bool SPLIT>
+// grid (d / 128 / CPC, slices).  partial [slice][128 tokens][d].  A CTA owns CPC adjacent tiles of
+// 128 output columns, which share every activation tile: these kernels are bound by the bytes the SMs
+// take in, from DRAM and L2 alike (about 6.5 TB/s in all), and with one column tile per CTA the
+// activation tiles that every CTA fetches again are as many bytes as the weights.
+template <bool SPLIT, int CPC>
 __global__ void __launch_bounds__(kMmaThreads, 1)
 ffn_down_swap_kernel(const __grid_constant__ CUtensorMap tm_wd, const __grid_constant__ CUtensorMap tm_act,
                      const __grid_constant__ CUtensorMap tm_act_lo, const int32_t *__restrict__ glist,
                      const int32_t *__restrict__ ng_dev, int N, int B, int d, int act_by_group,
                      float *__restrict__ partial, DeviceStatus *status) {
     extern __shared__ uint8_t smem_raw[];
-    const int c0 = blockIdx.x * 128, z = blockIdx.y, Z = gridDim.y;
+    const int c0 = blockIdx.x * 128 * CPC, z = blockIdx.y, Z = gridDim.y;
     const int ng = *ng_dev;
     const int gi0 = (int)(((long long)ng * z) / Z), gi1 = (int)(((long long)ng * (z + 1)) / Z);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -550,10 +553,10 @@ ffn_down_swap_kernel(const __grid_constant__ CUtensorMap tm_wd, const __grid_con
     Barriers *bars = reinterpret_cast<Barriers *>(base + kRingBytesMma);
     const int nblk = (N + 63) / 64;                                // token blocks of 64
     const int bbytes = nblk * 64 * BK * 2;                         // actT tile: 64 k rows x tokens
-    const int stage_bytes = kABytes + (SPLIT ? 2 : 1) * bbytes;
+    const int stage_bytes = CPC * kABytes + (SPLIT ? 2 : 1) * bbytes;
     const int stages = min(6, kRingBytesMma / stage_bytes);
     const int NB = SPLIT ? 2 * nblk * 64 : N;                      // MMA columns: value blocks then remainder blocks
-    const uint32_t tcols = NB <= 128 ? 128u : 256u;
+    const uint32_t tcols = CPC * NB <= 128 ? 128u : CPC * NB <= 256 ? 256u : 512u;
     setup_cta(bars, warp, tcols);
     const int kblocks = (gi1 - gi0) * 2;
 
@@ -567,11 +570,12 @@ ffn_down_swap_kernel(const __grid_constant__ CUtensorMap tm_wd, const __grid_con
                 const int arow = (act_by_group ? glist[gi] : gi) * 128 + half * BK;
                 uint8_t *st = base + (size_t)s * stage_bytes;
                 mbar_expect_tx(&bars->full[s], stage_bytes);
-                tma_load_2d(st, &tm_wd, c0, wrow, &bars->full[s]);
-                tma_load_2d(st + 64 * BK * 2, &tm_wd, c0 + 64, wrow, &bars->full[s]);
+#pragma unroll
+                for (int j = 0; j < 2 * CPC; ++j)   // weight tile of column tile j / 2: two blocks of 64 columns
+                    tma_load_2d(st + j * (64 * BK * 2), &tm_wd, c0 + j * 64, wrow, &bars->full[s]);
                 for (int i = 0; i < nblk; ++i) {
-                    tma_load_2d(st + kABytes + i * (64 * BK * 2), &tm_act, i * 64, arow, &bars->full[s]);
-                    if (SPLIT) tma_load_2d(st + kABytes + bbytes + i * (64 * BK * 2), &tm_act_lo, i * 64, arow, &bars->full[s]);
+                    tma_load_2d(st + CPC * kABytes + i * (64 * BK * 2), &tm_act, i * 64, arow, &bars->full[s]);
+                    if (SPLIT) tma_load_2d(st + CPC * kABytes + bbytes + i * (64 * BK * 2), &tm_act_lo, i * 64, arow, &bars->full[s]);
                 }
             }
         }
@@ -585,40 +589,48 @@ ffn_down_swap_kernel(const __grid_constant__ CUtensorMap tm_wd, const __grid_con
                 ok = mbar_wait(&bars->full[s], (kb / stages) & 1, bars, status);
                 if (!ok) break;
                 tc_fence_after();
-                const uint32_t a0 = smem_u32(base + (size_t)s * stage_bytes), b0 = a0 + kABytes;
+                const uint32_t a0 = smem_u32(base + (size_t)s * stage_bytes), b0 = a0 + CPC * kABytes;
 #pragma unroll
-                for (int k4 = 0; k4 < BK / 16; ++k4)   // remainder blocks follow the value blocks: one operand
-                    tc_mma(tmem, desc_sw128(a0 + k4 * 2048, 64 * BK * 2), desc_sw128(b0 + k4 * 2048, 64 * BK * 2),
-                           idesc, (kb | k4) != 0);
+                for (int k4 = 0; k4 < BK / 16; ++k4) {   // remainder blocks follow the value blocks: one operand
+                    const uint64_t bd = desc_sw128(b0 + k4 * 2048, 64 * BK * 2);
+#pragma unroll
+                    for (int ct = 0; ct < CPC; ++ct)
+                        tc_mma(tmem + ct * NB, desc_sw128(a0 + ct * kABytes + k4 * 2048, 64 * BK * 2), bd, idesc, (kb | k4) != 0);
+                }
                 tc_commit(&bars->empty[s]);
             }
             if (ok) tc_commit(&bars->acc_ready);
         }
     } else {
-        const int q = warp & 3, col = c0 + q * 32 + lane;
-        float *dst = partial + (size_t)z * 128 * d + col;
+        const int q = warp & 3;
         if (kblocks == 0) {
-            for (int tkn = 0; tkn < B; ++tkn) dst[(size_t)tkn * d] = 0.f;
+            for (int ct = 0; ct < CPC; ++ct) {
+                float *dst = partial + (size_t)z * 128 * d + c0 + ct * 128 + q * 32 + lane;
+                for (int tkn = 0; tkn < B; ++tkn) dst[(size_t)tkn * d] = 0.f;
+            }
         } else if (mbar_wait(&bars->acc_ready, 0, bars, status)) {
             tc_fence_after();
-            const uint32_t tbase = bars->tmem_base + ((uint32_t)(q * 32) << 16);
+            for (int ct = 0; ct < CPC; ++ct) {
+                const uint32_t tbase = bars->tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(ct * NB);
+                float *dst = partial + (size_t)z * 128 * d + c0 + ct * 128 + q * 32 + lane;
 #pragma unroll 1
-            for (int c = 0; c < N / 16; ++c) {
-                uint32_t v[16];
-                tc_ld16(tbase + c * 16, v);
-                if (SPLIT) {
-                    uint32_t v2[16];
-                    tc_ld16(tbase + nblk * 64 + c * 16, v2);
-                    tc_wait_ld();
+                for (int c = 0; c < N / 16; ++c) {
+                    uint32_t v[16];
+                    tc_ld16(tbase + c * 16, v);
+                    if (SPLIT) {
+                        uint32_t v2[16];
+                        tc_ld16(tbase + nblk * 64 + c * 16, v2);
+                        tc_wait_ld();
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) v[j] = __float_as_uint(__uint_as_float(v[j]) + __uint_as_float(v2[j]));
-                } else {
-                    tc_wait_ld();
-                }
+                        for (int j = 0; j < 16; ++j) v[j] = __float_as_uint(__uint_as_float(v[j]) + __uint_as_float(v2[j]));
+                    } else {
+                        tc_wait_ld();
+                    }
 #pragma unroll
-                for (int j = 0; j < 16; ++j) {
-                    const int tkn = c * 16 + j;
-                    if (tkn < B) dst[(size_t)tkn * d] = __uint_as_float(v[j]);
+                    for (int j = 0; j < 16; ++j) {
+                        const int tkn = c * 16 + j;
+                        if (tkn < B) dst[(size_t)tkn * d] = __uint_as_float(v[j]);
+                    }
                 }
             }
         }
@@ -816,7 +828,7 @@ cs_status prepare_ffn_mma(cs_plan *plan) {
     CS_CUDA_TRY(plan, cudaFuncSetAttribute(ffn_down_mma_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMmaSmem));
     CS_CUDA_TRY(plan, cudaFuncSetAttribute(ffn_down_mma_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMmaSmem));
     CS_CUDA_TRY(plan, cudaFuncSetAttribute(ffn_gateup_swap_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMmaSmem));
-    CS_CUDA_TRY(plan, cudaFuncSetAttribute(ffn_down_swap_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMmaSmem));
+    CS_CUDA_TRY(plan, cudaFuncSetAttribute(ffn_down_swap_kernel<true, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMmaSmem));
     return CS_OK;
 }
 
@@ -946,10 +958,10 @@ cs_status launch_decode_down(cs_plan *plan, const cs_layer *L, int B, bool act_b
     const int N = (B + 15) / 16 * 16;
     CUtensorMap tm[7];
     if (!decode_maps(plan, L, nullptr, nullptr, B, N, tm)) return record_cuda(plan, cudaErrorInvalidValue, "cuTensorMapEncodeTiled");
-    const int Z = max(1, min(plan->sm_count / (c.d / 128), 8));
+    const int Z = max(1, min(plan->sm_count / (c.d / 256), 8));   // two column tiles per CTA (d is a multiple of 256)
     {
         StageTimer timer(plan, CS_STAGE_EXEC2, st);
-        ffn_down_swap_kernel<true><<<dim3(c.d / 128, Z), kMmaThreads, kMmaSmem, st>>>(
+        ffn_down_swap_kernel<true, 2><<<dim3(c.d / 256, Z), kMmaThreads, kMmaSmem, st>>>(
             tm[4], tm[5], tm[6], plan->glist, plan->nu, N, B, c.d, act_by_group ? 1 : 0, plan->mma_partial, plan->status);
         plan->launches++;
         CS_CUDA_TRY(plan, cudaGetLastError());
