@@ -242,12 +242,21 @@ def run_ours(args):
         run_host(min(Wm, chunk))
         ms_e2e = timed(run_host, K)
 
-        # ---- per-stage device times (separate pass, events around every stage's launches)
+        # ---- per-stage device times: a separate pass with events around every stage's launches.  Each
+        # step is replayed from a one-step CUDA graph, in which the records are event nodes: a record
+        # issued from the host between two launches would add several microseconds to every bracket.
         plan.enable_timing(True)
         n_prof = min(K, 200)
-        acc = [0.0, 0.0, 0.0, 0.0, 0.0]
+        n_graphs = min(n_layers * (1 if chained else 2), 32)
+        stage_graphs = []
+        for i in range(n_graphs):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=stream):
+                step(i)
+            stage_graphs.append(g)
+        acc = [0.0] * 5
         for i in range(n_prof + 3):
-            step(i)
+            stage_graphs[i % n_graphs].replay()
             t = plan.stage_times(stream)
             if i >= 3:
                 acc = [a + b for a, b in zip(acc, t)]

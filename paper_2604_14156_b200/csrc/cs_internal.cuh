@@ -78,14 +78,23 @@ cs_status record_cuda(cs_plan *plan, cudaError_t e, const char *what);
         if (e_ != cudaSuccess) return ::cs::record_cuda((plan), e_, #expr);         \
     } while (0)
 
-// Brackets one stage's launches with events when timing is enabled.
+// Brackets one stage's launches with events when timing is enabled.  On a capturing stream the
+// records become event-record nodes of the graph (external events), which can be timed after a
+// replay and cost far less than a record issued from the host between two launches.
 struct StageTimer {
     cs_plan *p; int stage; cudaStream_t st;
+    static void record(cudaEvent_t ev, cudaStream_t s) {
+        cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+        if (cudaStreamIsCapturing(s, &cap) == cudaSuccess && cap == cudaStreamCaptureStatusActive)
+            cudaEventRecordWithFlags(ev, s, cudaEventRecordExternal);
+        else
+            cudaEventRecord(ev, s);
+    }
     StageTimer(cs_plan *plan, int s, cudaStream_t stream) : p(plan), stage(s), st(stream) {
-        if (p->timing) cudaEventRecord(p->ev[2 * stage], st);
+        if (p->timing) record(p->ev[2 * stage], st);
     }
     ~StageTimer() {
-        if (p->timing) { cudaEventRecord(p->ev[2 * stage + 1], st); p->stage_seen[stage] = 1; }
+        if (p->timing) { record(p->ev[2 * stage + 1], st); p->stage_seen[stage] = 1; }
     }
 };
 
