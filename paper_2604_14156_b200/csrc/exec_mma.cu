@@ -409,6 +409,112 @@ ffn_down_mma_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_con
 }
 
 
+// ---- down, one slice, tiles of 128 tokens x 320 columns -----------------------------------------------
+// With one list slice the number of tiles decides how evenly the SMs are loaded: 2048 tokens x 5120
+// columns are 320 tiles of 256 columns, 2.16 per SM, i.e. three rounds; tiles of 320 columns are 256,
+// two rounds of 1.25 times the work.  The accumulator takes 320 of the 512 tensor-memory columns and
+// every k step is two instructions (256 + 64 columns).  Activations bf16 (no remainder operand); the
+// epilogue writes the output itself.  grid (d / 320, token tiles).
+constexpr int BNW = 320;
+constexpr int kWideStage = kABytes + BNW * BK * 2;       // 16 KB + 40 KB
+constexpr int kWideStages = kRingBytesMma / kWideStage;  // 3
+
+__global__ void __launch_bounds__(kMmaThreads, 1)
+ffn_down_wide_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant__ CUtensorMap tm_wd,
+                     const int32_t *__restrict__ glist, const int32_t *__restrict__ ng_dev, int ng_host, int M, int d,
+                     const float *residual, float *out_f32, __nv_bfloat16 *__restrict__ out_bf16, DeviceStatus *status) {
+    extern __shared__ uint8_t smem_raw[];
+    const int nt = blockIdx.x, mt = blockIdx.y;
+    const int ng = ng_dev != nullptr ? *ng_dev : ng_host;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    uint8_t *base = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    Barriers *bars = reinterpret_cast<Barriers *>(base + kRingBytesMma);
+    setup_cta(bars, warp, 512);
+    const int kblocks = ng * 2;   // two 64-row k blocks per 128-channel group
+
+    if (warp == 0) {
+        if (lane == 0) {
+            for (int kb = 0; kb < kblocks; ++kb) {
+                const int s = kb % kWideStages;
+                if (kb >= kWideStages && !mbar_wait(&bars->empty[s], ((kb / kWideStages) - 1) & 1, bars, status)) break;
+                const int gi = kb >> 1, half = kb & 1;
+                const int wrow = glist[gi] * 128 + half * BK;
+                uint8_t *st = base + (size_t)s * kWideStage;
+                mbar_expect_tx(&bars->full[s], kWideStage);
+                tma_load_2d(st, &tm_act, gi * 128 + half * BK, mt * BM, &bars->full[s]);
+#pragma unroll
+                for (int j = 0; j < BNW / 64; ++j)
+                    tma_load_2d(st + kABytes + j * (64 * BK * 2), &tm_wd, nt * BNW + j * 64, wrow, &bars->full[s]);
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0 && kblocks > 0) {
+            const uint32_t idesc256 = make_idesc_rt(256, false, true), idesc64 = make_idesc_rt(64, false, true);
+            const uint32_t tmem = bars->tmem_base;
+            bool ok = true;
+            for (int kb = 0; kb < kblocks && ok; ++kb) {
+                const int s = kb % kWideStages;
+                ok = mbar_wait(&bars->full[s], (kb / kWideStages) & 1, bars, status);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t a0 = smem_u32(base + (size_t)s * kWideStage), b0 = a0 + kABytes;
+#pragma unroll
+                for (int k4 = 0; k4 < BK / 16; ++k4) {
+                    const uint64_t ad = desc_sw128(a0 + k4 * 32, 16);
+                    tc_mma(tmem, ad, desc_sw128(b0 + k4 * 2048, 64 * BK * 2), idesc256, (kb | k4) != 0);
+                    tc_mma(tmem + 256, ad, desc_sw128(b0 + 4 * (64 * BK * 2) + k4 * 2048, 64 * BK * 2), idesc64, (kb | k4) != 0);
+                }
+                tc_commit(&bars->empty[s]);
+            }
+            if (ok) tc_commit(&bars->acc_ready);
+        }
+    } else {
+        const int q = warp & 3;
+        const int m = mt * BM + q * 32 + lane;
+        if (kblocks > 0 && mbar_wait(&bars->acc_ready, 0, bars, status)) {
+            tc_fence_after();
+            const uint32_t tbase = bars->tmem_base + ((uint32_t)(q * 32) << 16);
+            const size_t o = (size_t)m * d + (size_t)nt * BNW;
+#pragma unroll 1
+            for (int c = 0; c < BNW / 32; ++c) {
+                uint32_t v[32];
+                tc_ld32(tbase + c * 32, v);
+                tc_wait_ld();
+                if (m < M) {
+                    if (residual != nullptr) {
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) {
+                            const float4 r = *reinterpret_cast<const float4 *>(residual + o + c * 32 + 4 * j);
+                            v[4 * j] = __float_as_uint(__uint_as_float(v[4 * j]) + r.x);
+                            v[4 * j + 1] = __float_as_uint(__uint_as_float(v[4 * j + 1]) + r.y);
+                            v[4 * j + 2] = __float_as_uint(__uint_as_float(v[4 * j + 2]) + r.z);
+                            v[4 * j + 3] = __float_as_uint(__uint_as_float(v[4 * j + 3]) + r.w);
+                        }
+                    }
+                    if (out_f32 != nullptr) {
+#pragma unroll
+                        for (int j = 0; j < 8; ++j)
+                            *reinterpret_cast<uint4 *>(out_f32 + o + c * 32 + 4 * j) = make_uint4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            uint32_t pk[4];
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                const __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(v[8 * j + 2 * e]), __uint_as_float(v[8 * j + 2 * e + 1]));
+                                pk[e] = *reinterpret_cast<const uint32_t *>(&h2);
+                            }
+                            *reinterpret_cast<uint4 *>(out_bf16 + o + c * 32 + 8 * j) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                        }
+                    }
+                }
+            }
+        }
+    }
+    teardown_cta(bars, warp, 512);
+}
+
+
 // ---- decode batches of at most 128 tokens: weights on the M side -------------------------------
 // With few tokens the cheap orientation is the transposed one: the 128 channel rows of a weight
 // block are the MMA's M operand and the tokens its N columns (N = batch rounded up to 16), so an
@@ -823,6 +929,7 @@ bool make_map(CUtensorMap *map, const void *base, uint64_t inner, uint64_t outer
 }  // namespace
 
 cs_status prepare_ffn_mma(cs_plan *plan) {
+    CS_CUDA_TRY(plan, cudaFuncSetAttribute(ffn_down_wide_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMmaSmem));
     CS_CUDA_TRY(plan, cudaFuncSetAttribute(ffn_gateup_mma_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMmaSmem));
     CS_CUDA_TRY(plan, cudaFuncSetAttribute(ffn_gateup_mma_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMmaSmem));
     CS_CUDA_TRY(plan, cudaFuncSetAttribute(ffn_down_mma_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMmaSmem));
@@ -877,7 +984,14 @@ cs_status launch_ffn_mma(cs_plan *plan, const cs_layer *L, const void *X, const 
         const int ntiles = c.d / BN;
         int Z = 1;
         if (mtiles * ntiles < plan->sm_count) Z = max(1, min(plan->sm_count / (mtiles * ntiles), plan->mma_slices));
-        if (split)
+        // one slice, bf16 activations: tiles of 320 columns when they need fewer rounds over the SMs
+        const int sms = plan->sm_count;
+        const bool wide = !split && Z == 1 && c.d % BNW == 0 && ng_host > 0 &&
+                          ((mtiles * (c.d / BNW) + sms - 1) / sms) * BNW < ((mtiles * ntiles + sms - 1) / sms) * BN;
+        if (wide)
+            ffn_down_wide_kernel<<<dim3(c.d / BNW, mtiles), kMmaThreads, kMmaSmem, st>>>(
+                tm_act, tm_wd, glist, ng_dev, ng_host, M, c.d, residual, out_f32, static_cast<__nv_bfloat16 *>(out_bf16), plan->status);
+        else if (split)
             ffn_down_mma_kernel<true><<<dim3(ntiles, mtiles, Z), kMmaThreads, kMmaSmem, st>>>(
                 tm_act, tm_act_lo, tm_wd, glist, ng_dev, ng_host, M, m_pad, c.d, plan->mma_partial, residual, out_f32,
                 static_cast<__nv_bfloat16 *>(out_bf16), plan->status);
