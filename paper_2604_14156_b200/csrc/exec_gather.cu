@@ -109,25 +109,37 @@ ffn_gather_kernel(const WT *__restrict__ Wg, const WT *__restrict__ Wu, const WT
 #pragma unroll
     for (int i = 0; i < kUnitStages; ++i) issue_unit(i);
     int stage = 0;
+    // When the number of segments divides the number of warps, a warp meets the same segment in every
+    // unit and its slice of h is loaded once; otherwise it is fetched (from L1) per unit.
+    const bool fixed_seg = kGatherWarps % nseg == 0;
+    float hv[kUnitChunks][E];
+    auto load_h = [&](int seg) {
+        const float *hp = h_lane + seg * kSegElems;
+#pragma unroll
+        for (int j = 0; j < kUnitChunks; ++j) {
+#pragma unroll
+            for (int e = 0; e < E; e += 4) {
+                float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (FULL || (seg * kUnitChunks + j) * 32 + lane < chunks) v = __ldg(reinterpret_cast<const float4 *>(hp + j * 32 * E + e));
+                hv[j][e] = v.x; hv[j][e + 1] = v.y; hv[j][e + 2] = v.z; hv[j][e + 3] = v.w;
+            }
+        }
+    };
+    if (fixed_seg) load_h(cc.seg);
 #pragma unroll 1
     for (; cc.u < nunits; advance(cc)) {
+        if (!fixed_seg) load_h(cc.seg);
         cp_async_wait<kUnitStages - 1>();
         const uint4 *src = wring + stage * (2 * kUnitChunks * 32);
-        const float *hp = h_lane + cc.seg * kSegElems;
         float g = 0.f, up = 0.f;
 #pragma unroll
         for (int j = 0; j < kUnitChunks; ++j) {
             if (FULL || (cc.seg * kUnitChunks + j) * 32 + lane < chunks) {
-                float hv[E], wg[E], wu[E];
-#pragma unroll
-                for (int e = 0; e < E; e += 4) {
-                    const float4 v = __ldg(reinterpret_cast<const float4 *>(hp + j * 32 * E + e));
-                    hv[e] = v.x; hv[e + 1] = v.y; hv[e + 2] = v.z; hv[e + 3] = v.w;
-                }
+                float wg[E], wu[E];
                 Chunk<WT>::widen(src[j * 32], wg);
                 Chunk<WT>::widen(src[(kUnitChunks + j) * 32], wu);
 #pragma unroll
-                for (int e = 0; e < E; ++e) { g = fmaf(wg[e], hv[e], g); up = fmaf(wu[e], hv[e], up); }
+                for (int e = 0; e < E; ++e) { g = fmaf(wg[e], hv[j][e], g); up = fmaf(wu[e], hv[j][e], up); }
             }
         }
         issue_unit(stage);  // refill the stage just consumed (its values were used above)
