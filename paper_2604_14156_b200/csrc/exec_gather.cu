@@ -212,15 +212,19 @@ ffn_gather_kernel(const WT *__restrict__ Wg, const WT *__restrict__ Wu, const WT
 }
 
 // out[t, :] = residual[t, :] + sum_{p < nx} partial[t, p, :], p ascending within fixed groups.
-// CTA = 32 float4 columns x kReduceGroups partial groups; a thread sums the partials p with
+// CTA = kReduceCols float4 columns x kReduceGroups partial groups; a thread sums the partials p with
 // p % kReduceGroups == its group, then the groups are folded in index order through shared memory.
-__global__ void __launch_bounds__(32 * kReduceGroups)
+// Small CTAs (256 threads, few registers) on purpose: under programmatic dependent launch they fit
+// on the SMs beside the gather kernel's CTAs and are in place when its last partial lands.
+constexpr int kReduceCols = 8;
+__global__ void __launch_bounds__(kReduceCols * kReduceGroups)
 reduce_partials_kernel(const float *__restrict__ partial, int nx, int d, const float *__restrict__ residual,
                        float *__restrict__ out) {
-    __shared__ float4 fold[kReduceGroups][32];
+    __shared__ float4 fold[kReduceGroups][kReduceCols];
     const int t = blockIdx.y;
-    const int col = blockIdx.x * 32 + (threadIdx.x & 31);  // float4 column
-    const int grp = threadIdx.x >> 5;
+    const int cl = threadIdx.x & (kReduceCols - 1);
+    const int col = blockIdx.x * kReduceCols + cl;          // float4 column
+    const int grp = threadIdx.x / kReduceCols;
     const int cols = d >> 2;
     pdl_launch_dependents();
     pdl_wait();
@@ -243,14 +247,14 @@ reduce_partials_kernel(const float *__restrict__ partial, int nx, int d, const f
             s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
         }
     }
-    fold[grp][threadIdx.x & 31] = s;
+    fold[grp][cl] = s;
     __syncthreads();
     if (grp == 0 && col < cols) {
         float4 r = residual != nullptr ? reinterpret_cast<const float4 *>(residual + (size_t)t * d)[col]
                                        : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
         for (int g = 0; g < kReduceGroups; ++g) {
-            const float4 v = fold[g][threadIdx.x & 31];
+            const float4 v = fold[g][cl];
             r.x += v.x; r.y += v.y; r.z += v.z; r.w += v.w;
         }
         reinterpret_cast<float4 *>(out + (size_t)t * d)[col] = r;
@@ -316,10 +320,10 @@ static cs_status gather_typed(cs_plan *plan, const cs_layer *L, const float *h, 
         }
         plan->launches++;
         CS_CUDA_TRY(plan, cudaGetLastError());
-        dim3 rgrid((c.d / 4 + 31) / 32, nb);
+        dim3 rgrid((c.d / 4 + kReduceCols - 1) / kReduceCols, nb);
         {
             StageTimer timer(plan, CS_STAGE_REDUCE, st);
-            launch_pdl(true, reduce_partials_kernel, rgrid, dim3(32 * kReduceGroups), 0, st, (const float *)plan->partial, nx,
+            launch_pdl(true, reduce_partials_kernel, rgrid, dim3(kReduceCols * kReduceGroups), 0, st, (const float *)plan->partial, nx,
                        c.d, residual ? residual + (size_t)t0 * c.d : (const float *)nullptr, out + (size_t)t0 * c.d);
         }
         plan->launches++;
@@ -399,8 +403,8 @@ static cudaError_t static_launch(const cs_config &c, const cs_layer *L, const fl
     launch_gather_kernel<WT>(grid, st, cpt, c.d / E, Wg, Wu, Wd, h, support, c.d, c.group, c.k, partial);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    dim3 rgrid((c.d / 4 + 31) / 32, B);
-    reduce_partials_kernel<<<rgrid, 32 * kReduceGroups, 0, st>>>(partial, nx, c.d, residual, out);
+    dim3 rgrid((c.d / 4 + kReduceCols - 1) / kReduceCols, B);
+    reduce_partials_kernel<<<rgrid, kReduceCols * kReduceGroups, 0, st>>>(partial, nx, c.d, residual, out);
     return cudaGetLastError();
 }
 
