@@ -142,9 +142,11 @@ static bool use_decode_mma(const cs_plan *plan, int B) { return plan->mma_ok && 
 // sizes the union of the supports is, to within a group or two, every group), so it runs on the
 // caller's stream while `side_work` -- sketch / recovery / bucketing -- runs on the plan's second
 // stream; the two join before the activations are masked and the down GEMM starts.
+// gamma != NULL: h is the un-normalised x and the operand split applies the RMSNorm itself.
 template <typename SideWork>
 static cs_status exec_decode_overlapped(cs_plan *plan, const cs_layer *layer, const float *h, int B,
-                                        const float *residual, float *out, cudaStream_t st, SideWork side_work) {
+                                        const float *residual, float *out, cudaStream_t st, SideWork side_work,
+                                        const float *gamma = nullptr) {
     __nv_bfloat16 *x_hi = static_cast<__nv_bfloat16 *>(plan->x_bf16);
     __nv_bfloat16 *x_lo = x_hi + (size_t)plan->cfg.max_tokens * plan->cfg.d;
     CS_CUDA_TRY(plan, cudaEventRecord(plan->ev_fork, st));
@@ -153,7 +155,8 @@ static cs_status exec_decode_overlapped(cs_plan *plan, const cs_layer *layer, co
     if (s != CS_OK) return s;
     CS_CUDA_TRY(plan, cudaEventRecord(plan->ev_join, plan->side));
     // f32 activations go in as two bf16 parts so that the result keeps f32-level accuracy
-    s = launch_split_bf16(plan, h, x_hi, x_lo, (size_t)B * plan->cfg.d, st);
+    s = gamma != nullptr ? launch_norm_split_bf16(plan, h, gamma, B, x_hi, x_lo, st)
+                         : launch_split_bf16(plan, h, x_hi, x_lo, (size_t)B * plan->cfg.d, st);
     if (s != CS_OK) return s;
     s = launch_decode_gateup(plan, layer, x_hi, x_lo, B, false, st);
     if (s != CS_OK) return s;
@@ -222,19 +225,16 @@ cs_status cs_layer_step(cs_plan *plan, const cs_layer *layer, const float *x, in
     const float *n = norm ? plan->n_buf : x;
     int32_t *sup = support_out != nullptr ? support_out : plan->sup_buf;
     if (use_decode_mma(plan, B)) {
-        // recovery (and, without a normalisation to wait for, the sketch too) beside the gate/up GEMM
-        if (norm) {
-            s = launch_sketch(plan, layer->S, x, layer->rms_gamma, B, plan->y_buf, plan->n_buf, layer->Phi, layer->mu, st);
-            if (s != CS_OK) return s;
-        }
-        return exec_decode_overlapped(plan, layer, n, B, layer->add_residual ? x : nullptr, x_out, st,
+        // sketch, recovery and bucketing run beside the gate/up GEMM; with a normalisation the GEMM's
+        // operand split normalises for itself, so that it does not wait for the sketch kernel either
+        return exec_decode_overlapped(plan, layer, x, B, layer->add_residual ? x : nullptr, x_out, st,
                                       [&](cudaStream_t side) {
-            cs_status r = CS_OK;
-            if (!norm) r = launch_sketch(plan, layer->S, x, nullptr, B, plan->y_buf, nullptr, layer->Phi, layer->mu, side);
+            cs_status r = launch_sketch(plan, layer->S, x, layer->rms_gamma, B, plan->y_buf, norm ? plan->n_buf : nullptr,
+                                        layer->Phi, layer->mu, side);
             if (r == CS_OK) r = launch_recover(plan, layer->Phi, layer->mu, plan->y_buf, B, sup, z_out, resid_out, true, side);
             if (r == CS_OK) r = launch_bucket(plan, sup, B, side);
             return r;
-        });
+        }, layer->rms_gamma);
     }
     s = launch_sketch(plan, layer->S, x, layer->rms_gamma, B, plan->y_buf, norm ? plan->n_buf : nullptr, layer->Phi, layer->mu, st);
     if (s != CS_OK) return s;

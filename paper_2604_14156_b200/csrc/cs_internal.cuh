@@ -113,6 +113,8 @@ cs_status prepare_ffn_mma(cs_plan *plan);
 cs_status launch_bucket(cs_plan *plan, const int32_t *support, int B, cudaStream_t st, int32_t *counts = nullptr,
                         int32_t *offsets = nullptr, int32_t *token_ids = nullptr);
 cs_status launch_split_bf16(cs_plan *plan, const float *x, void *y_hi, void *y_lo, size_t n, cudaStream_t st);
+cs_status launch_norm_split_bf16(cs_plan *plan, const float *x, const float *gamma, int B, void *y_hi, void *y_lo,
+                                 cudaStream_t st);
 cs_status launch_ffn_mma(cs_plan *plan, const cs_layer *L, const void *X, const void *X_lo, int M, const int32_t *glist,
                          const int32_t *ng_dev, int ng_host, const uint32_t *mask, const float *residual,
                          float *out_f32, void *out_bf16, cudaStream_t st);

@@ -806,6 +806,44 @@ __global__ void split_bf16_kernel(const float *__restrict__ x, __nv_bfloat16 *__
     reinterpret_cast<uint2 *>(y_lo)[i] = q;
 }
 
+// The same with the RMSNorm of the stacked workload in front: n = x * rsqrt(mean(x^2) + eps) * gamma,
+// one CTA per token.  The GEMM's operand does not have to wait for the sketch kernel, which forms the
+// same n for itself on the other stream.
+constexpr int kNormSplitThreads = 256;
+__global__ void __launch_bounds__(kNormSplitThreads)
+norm_split_bf16_kernel(const float *__restrict__ x, const float *__restrict__ gamma, float eps, int d,
+                       __nv_bfloat16 *__restrict__ y_hi, __nv_bfloat16 *__restrict__ y_lo) {
+    __shared__ float red[kNormSplitThreads / 32];
+    const int t = blockIdx.x, tid = threadIdx.x;
+    const float4 *xr = reinterpret_cast<const float4 *>(x + (size_t)t * d);
+    const float4 *gr = reinterpret_cast<const float4 *>(gamma);
+    float ss = 0.f;
+    for (int c = tid; c < d / 4; c += kNormSplitThreads) {
+        const float4 v = xr[c];
+        ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+    }
+    ss = warp_sum(ss);
+    if ((tid & 31) == 0) red[tid >> 5] = ss;
+    __syncthreads();
+    float tot = 0.f;
+#pragma unroll
+    for (int w = 0; w < kNormSplitThreads / 32; ++w) tot += red[w];
+    const float rscale = rsqrtf(tot / (float)d + eps);
+    for (int c = tid; c < d / 4; c += kNormSplitThreads) {
+        float4 v = xr[c];
+        const float4 g = gr[c];
+        v.x = v.x * g.x * rscale; v.y = v.y * g.y * rscale; v.z = v.z * g.z * rscale; v.w = v.w * g.w * rscale;
+        const __nv_bfloat162 h0 = __floats2bfloat162_rn(v.x, v.y), h1 = __floats2bfloat162_rn(v.z, v.w);
+        const __nv_bfloat162 l0 = __floats2bfloat162_rn(v.x - __low2float(h0), v.y - __high2float(h0));
+        const __nv_bfloat162 l1 = __floats2bfloat162_rn(v.z - __low2float(h1), v.w - __high2float(h1));
+        uint2 p, q;
+        p.x = *reinterpret_cast<const uint32_t *>(&h0); p.y = *reinterpret_cast<const uint32_t *>(&h1);
+        q.x = *reinterpret_cast<const uint32_t *>(&l0); q.y = *reinterpret_cast<const uint32_t *>(&l1);
+        reinterpret_cast<uint2 *>(y_hi + (size_t)t * d)[c] = p;
+        reinterpret_cast<uint2 *>(y_lo + (size_t)t * d)[c] = q;
+    }
+}
+
 // ---- bucketing: supports [B,k] -> membership masks, per-group token lists, union list ------------
 // One CTA.  mask [B][4] (bit g of token t), counts [G], offsets [G+1], token_ids [B*k] (tokens of
 // group g ascending at offsets[g]..offsets[g+1]), glist [G] (groups with a non-empty bucket,
@@ -1087,6 +1125,15 @@ cs_status launch_decode_down(cs_plan *plan, const cs_layer *L, int B, bool act_b
         plan->launches++;
         CS_CUDA_TRY(plan, cudaGetLastError());
     }
+    return CS_OK;
+}
+
+cs_status launch_norm_split_bf16(cs_plan *plan, const float *x, const float *gamma, int B, void *y_hi, void *y_lo,
+                                 cudaStream_t st) {
+    norm_split_bf16_kernel<<<B, kNormSplitThreads, 0, st>>>(x, gamma, plan->cfg.rms_eps, plan->cfg.d,
+                                                            static_cast<__nv_bfloat16 *>(y_hi), static_cast<__nv_bfloat16 *>(y_lo));
+    plan->launches++;
+    CS_CUDA_TRY(plan, cudaGetLastError());
     return CS_OK;
 }
 
