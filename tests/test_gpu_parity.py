@@ -115,6 +115,40 @@ def test_recover_ties_across_warps(name, k):
             assert np.array_equal(sup1[t].cpu().numpy(), one.support), t
 
 
+def test_recover_random_shapes():
+    """Forty random (G, m, k, T) shapes, all warp counts and both forms of the kernel (list for
+    k <= 56, dense above), some with duplicated columns or an all-zero sketch."""
+    rs = np.random.default_rng(7)
+    excused = total = 0
+    for trial in range(40):
+        G = int(rs.integers(2, 129)); m = int(rs.integers(2, 65)); k = int(rs.integers(1, G + 1)); T = int(rs.integers(0, 31))
+        if trial % 5 == 0 and G >= 57:
+            k = int(rs.integers(57, G + 1))
+        B = 4
+        Phi = torch.tensor(rs.normal(0, m ** -0.5, (m, G)), dtype=torch.float32)
+        if trial % 7 == 0 and G > 40:
+            Phi[:, 33] = Phi[:, 1]; Phi[:, 7] = -Phi[:, 6]
+        mu = W.spectral_step(Phi)
+        y = torch.tensor(rs.normal(size=(B, m)), dtype=torch.float32)
+        if trial % 11 == 0:
+            y[0] = 0
+        plan = cs.Plan(256, G * 64, 64, m, k, T, torch.float32, B, 1e-5)
+        sup, z, resid = cs.cs_recover(plan, Phi.to(DEV), mu, y.to(DEV))
+        sup = sup.cpu().numpy(); z = z.cpu().numpy(); resid = resid.cpu().numpy()
+        for t in range(B):
+            ref = oracle.iht(Phi, y[t], k, T, mu)
+            total += 1
+            if np.array_equal(sup[t], ref.support):
+                zr = ref.z[ref.support]
+                assert (rel(z[t], zr) <= Z_TOL) if zr.any() else not z[t].any(), (G, m, k, T, t)
+                assert abs(resid[t] - ref.resid) <= 1e-4 * max(1.0, ref.resid), (G, m, k, T, t)
+            else:
+                assert ref.min_gap <= GAP_TOL, (G, m, k, T, t, ref.min_gap)
+                excused += 1
+        plan.close()
+    assert excused <= total // 20
+
+
 @pytest.mark.parametrize("name,B", [("tiny_f32", 4), ("l2_7b_b1", 1), ("l2_7b_b64", 3)])
 def test_ffn_exec_matches_oracle_on_given_supports(name, B):
     cfg = W.CONFIGS[name]
