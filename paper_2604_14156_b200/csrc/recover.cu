@@ -68,6 +68,14 @@ recover_kernel(const float *__restrict__ Phi, const float *__restrict__ gram, fl
     const bool valid = g < G;
     const int t = blockIdx.x;
     pdl_launch_dependents();
+    // Phi is a parameter: this thread's column (needed for c) is requested before the wait for the
+    // kernel that produces y and M, when it fits 32 registers
+    const bool early_phi = m <= 32;
+    float phc[32];
+    if (early_phi) {
+#pragma unroll
+        for (int row = 0; row < 32; ++row) phc[row] = (valid && row < m) ? __ldg(Phi + row * G + g) : 0.f;
+    }
     pdl_wait();   // y and M come from the kernel before
     float mreg[NR];
     if constexpr (KC == 0) {   // row g of M (M is symmetric: row g is the column that multiplies into entry g)
@@ -90,7 +98,17 @@ recover_kernel(const float *__restrict__ Phi, const float *__restrict__ gram, fl
     __syncthreads();
     // c_g = mu sum_i Phi[i,g] y_i
     float cg = 0.f;
-    if (valid) {
+    if (valid && early_phi) {
+        float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+#pragma unroll
+        for (int row = 0; row < 32; row += 4) {   // rows past m hold zeros
+            const float y0 = row < m ? y_s[row] : 0.f, y1 = row + 1 < m ? y_s[row + 1] : 0.f;
+            const float y2 = row + 2 < m ? y_s[row + 2] : 0.f, y3 = row + 3 < m ? y_s[row + 3] : 0.f;
+            a0 = fmaf(phc[row], y0, a0); a1 = fmaf(phc[row + 1], y1, a1);
+            a2 = fmaf(phc[row + 2], y2, a2); a3 = fmaf(phc[row + 3], y3, a3);
+        }
+        cg = mu * ((a0 + a1) + (a2 + a3));
+    } else if (valid) {
         float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
         const float *pcol = Phi + g;
         int row = 0;

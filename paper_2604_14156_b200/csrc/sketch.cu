@@ -35,6 +35,18 @@ sketch_kernel(const float *__restrict__ S, const float *__restrict__ x, const fl
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int chunks = d >> 2;
     pdl_launch_dependents();
+    // S is a parameter: with a single row per CTA (small batches) its chunks are requested before the
+    // wait for the kernel that produces x, which takes the DRAM latency of S off the chain.
+    const bool early = nrows == 1;
+    float4 s0[CPT];
+    if (early) {
+        const float4 *row = reinterpret_cast<const float4 *>(S + (size_t)r0 * d);
+#pragma unroll
+        for (int j = 0; j < CPT; ++j) {
+            const int c = tid + j * kSketchThreads;
+            s0[j] = c < chunks ? __ldg(row + c) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+    }
     pdl_wait();   // x may be the previous kernel's output
 
     float4 xv[CPT];
@@ -59,7 +71,7 @@ sketch_kernel(const float *__restrict__ S, const float *__restrict__ x, const fl
         for (int j = 0; j < CPT; ++j) {
             const int c = tid + j * kSketchThreads;
             if (c < chunks) {
-                const float4 s = __ldg(row + c);
+                const float4 s = early ? s0[j] : __ldg(row + c);
                 acc = fmaf(s.x, xv[j].x, acc); acc = fmaf(s.y, xv[j].y, acc);
                 acc = fmaf(s.z, xv[j].z, acc); acc = fmaf(s.w, xv[j].w, acc);
             }
