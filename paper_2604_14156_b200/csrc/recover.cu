@@ -78,6 +78,14 @@ recover_kernel(const float *__restrict__ Phi, const float *__restrict__ gram, fl
     }
     pdl_wait();   // y and M come from the kernel before
     float mreg[NR];
+    const float *mcol = gram + (valid ? g : 0);
+    if constexpr (KC > 0) {
+        // List form: the entries M[idx_j, g] that go with the list come straight from global memory (M is
+        // 30 to 60 KB and stays in L1/L2) and are fetched again only when the support changes, which
+        // keeps the CTA's shared memory at 2 KB.  The first list is 0..k-1: requested at once.
+#pragma unroll
+        for (int j = 0; j < NR; ++j) mreg[j] = __ldg(mcol + (j < k ? j : 0) * GP);
+    }
     if constexpr (KC == 0) {   // row g of M (M is symmetric: row g is the column that multiplies into entry g)
         const float4 *src = reinterpret_cast<const float4 *>(gram + (size_t)(valid ? g : 0) * GP);
 #pragma unroll
@@ -119,14 +127,6 @@ recover_kernel(const float *__restrict__ Phi, const float *__restrict__ gram, fl
         }
         for (; row < m; ++row) a0 = fmaf(__ldg(pcol + row * G), y_s[row], a0);
         cg = mu * ((a0 + a1) + (a2 + a3));
-    }
-    // List form: the entries M[idx_j, g] that go with the list come straight from global memory (M is
-    // 30 to 60 KB and stays in L1/L2) and are fetched again only when the support changes, which
-    // keeps the CTA's shared memory at 2 KB.
-    const float *mcol = gram + (valid ? g : 0);
-    if constexpr (KC > 0) {
-#pragma unroll
-        for (int j = 0; j < NR; ++j) mreg[j] = __ldg(mcol + idx_s[j] * GP);
     }
     const unsigned lt_mask = (1u << lane) - 1u;
     const int rank_total = G * (G - 1) / 2;   // what the ranks of G distinct positions add up to
