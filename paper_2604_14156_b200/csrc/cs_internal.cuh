@@ -136,6 +136,26 @@ inline bool pdl_for(const cs_plan *plan, int B) { return !(plan->mma_ok && B >= 
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
+// Loads of data that the kernel before this one produced.  They are volatile asm statements, like
+// the wait itself, so the compiler keeps them after it; a plain load through a const __restrict__
+// pointer (or __ldg) may be turned into a non-coherent load and moved above the wait, which reads
+// what the buffer held before (seen as rare wrong recoveries when a plan's scratch was reused).
+__device__ __forceinline__ float ld_dep(const float *p) {
+    float v;
+    asm volatile("ld.global.f32 %0, [%1];" : "=f"(v) : "l"(p));
+    return v;
+}
+__device__ __forceinline__ int ld_dep(const int32_t *p) {
+    int v;
+    asm volatile("ld.global.s32 %0, [%1];" : "=r"(v) : "l"(p));
+    return v;
+}
+__device__ __forceinline__ float4 ld_dep4(const float *p) {
+    float4 v;
+    asm volatile("ld.global.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(p));
+    return v;
+}
+
 template <typename... KArgs, typename... Args>
 inline cudaError_t launch_pdl(bool pdl, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
                               cudaStream_t st, Args... args) {

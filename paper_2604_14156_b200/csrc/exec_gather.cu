@@ -73,7 +73,7 @@ ffn_gather_kernel(const WT *__restrict__ Wg, const WT *__restrict__ Wu, const WT
 
     if (tid < nrows) {
         const int c = r_begin + tid;
-        chan_s[tid] = support[(size_t)t * k + c / b] * b + c % b;
+        chan_s[tid] = ld_dep(support + (size_t)t * k + c / b) * b + c % b;
     }
     __syncthreads();
 
@@ -120,7 +120,7 @@ ffn_gather_kernel(const WT *__restrict__ Wg, const WT *__restrict__ Wu, const WT
 #pragma unroll
             for (int e = 0; e < E; e += 4) {
                 float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-                if (FULL || (seg * kUnitChunks + j) * 32 + lane < chunks) v = __ldg(reinterpret_cast<const float4 *>(hp + j * 32 * E + e));
+                if (FULL || (seg * kUnitChunks + j) * 32 + lane < chunks) v = ld_dep4(hp + j * 32 * E + e);
                 hv[j][e] = v.x; hv[j][e + 1] = v.y; hv[j][e + 2] = v.z; hv[j][e + 3] = v.w;
             }
         }
@@ -234,23 +234,24 @@ reduce_partials_kernel(const float *__restrict__ partial, int nx, int d, const f
         // partials p = grp, grp + 32, ...: loads issued four at a time, added in index order
         int p = grp;
         for (; p + 3 * kReduceGroups < nx; p += 4 * kReduceGroups) {
-            const float4 v0 = src[(size_t)p * cols], v1 = src[(size_t)(p + kReduceGroups) * cols],
-                         v2 = src[(size_t)(p + 2 * kReduceGroups) * cols],
-                         v3 = src[(size_t)(p + 3 * kReduceGroups) * cols];
+            const float4 v0 = ld_dep4(reinterpret_cast<const float *>(src + (size_t)p * cols)),
+                         v1 = ld_dep4(reinterpret_cast<const float *>(src + (size_t)(p + kReduceGroups) * cols)),
+                         v2 = ld_dep4(reinterpret_cast<const float *>(src + (size_t)(p + 2 * kReduceGroups) * cols)),
+                         v3 = ld_dep4(reinterpret_cast<const float *>(src + (size_t)(p + 3 * kReduceGroups) * cols));
             s.x += v0.x; s.y += v0.y; s.z += v0.z; s.w += v0.w;
             s.x += v1.x; s.y += v1.y; s.z += v1.z; s.w += v1.w;
             s.x += v2.x; s.y += v2.y; s.z += v2.z; s.w += v2.w;
             s.x += v3.x; s.y += v3.y; s.z += v3.z; s.w += v3.w;
         }
         for (; p < nx; p += kReduceGroups) {
-            const float4 v = src[(size_t)p * cols];
+            const float4 v = ld_dep4(reinterpret_cast<const float *>(src + (size_t)p * cols));
             s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
         }
     }
     fold[grp][cl] = s;
     __syncthreads();
     if (grp == 0 && col < cols) {
-        float4 r = residual != nullptr ? reinterpret_cast<const float4 *>(residual + (size_t)t * d)[col]
+        float4 r = residual != nullptr ? ld_dep4(residual + (size_t)t * d + 4 * (size_t)col)
                                        : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
         for (int g = 0; g < kReduceGroups; ++g) {

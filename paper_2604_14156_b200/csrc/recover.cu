@@ -84,17 +84,17 @@ recover_kernel(const float *__restrict__ Phi, const float *__restrict__ gram, fl
         // 30 to 60 KB and stays in L1/L2) and are fetched again only when the support changes, which
         // keeps the CTA's shared memory at 2 KB.  The first list is 0..k-1: requested at once.
 #pragma unroll
-        for (int j = 0; j < NR; ++j) mreg[j] = __ldg(mcol + (j < k ? j : 0) * GP);
+        for (int j = 0; j < NR; ++j) mreg[j] = ld_dep(mcol + (j < k ? j : 0) * GP);
     }
     if constexpr (KC == 0) {   // row g of M (M is symmetric: row g is the column that multiplies into entry g)
-        const float4 *src = reinterpret_cast<const float4 *>(gram + (size_t)(valid ? g : 0) * GP);
+        const float *src = gram + (size_t)(valid ? g : 0) * GP;
 #pragma unroll
         for (int j = 0; j < GP / 4; ++j) {
-            const float4 q = __ldg(src + j);
+            const float4 q = ld_dep4(src + 4 * j);
             mreg[4 * j] = q.x; mreg[4 * j + 1] = q.y; mreg[4 * j + 2] = q.z; mreg[4 * j + 3] = q.w;
         }
     }
-    for (int row = tid; row < m; row += GP) y_s[row] = y[(size_t)t * m + row];
+    for (int row = tid; row < m; row += GP) y_s[row] = ld_dep(y + (size_t)t * m + row);
     // z_0 = 0 with the support the order assigns to an all-zero vector: indices 0..k-1
     for (int i = tid; i < NV; i += GP) {
         val_s[0][i] = 0.f; val_s[1][i] = 0.f;
@@ -194,7 +194,7 @@ recover_kernel(const float *__restrict__ Phi, const float *__restrict__ gram, fl
         __syncthreads();
         if constexpr (KC > 0) {
 #pragma unroll
-            for (int j = 0; j < NR; ++j) mreg[j] = __ldg(mcol + idx_s[j] * GP);
+            for (int j = 0; j < NR; ++j) mreg[j] = ld_dep(mcol + idx_s[j] * GP);
         }
     }
 

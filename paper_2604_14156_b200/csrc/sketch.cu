@@ -56,7 +56,7 @@ sketch_kernel(const float *__restrict__ S, const float *__restrict__ x, const fl
         const int c = tid + j * kSketchThreads;
         xv[j] = make_float4(0.f, 0.f, 0.f, 0.f);
         if (c < chunks) {
-            xv[j] = reinterpret_cast<const float4 *>(x + (size_t)t * d)[c];
+            xv[j] = ld_dep4(x + (size_t)t * d + 4 * (size_t)c);
             ss += xv[j].x * xv[j].x + xv[j].y * xv[j].y + xv[j].z * xv[j].z + xv[j].w * xv[j].w;
             if (gamma != nullptr) {
                 const float4 g = reinterpret_cast<const float4 *>(gamma)[c];

@@ -116,11 +116,11 @@ def test_recover_ties_across_warps(name, k):
 
 
 def test_recover_random_shapes():
-    """Forty random (G, m, k, T) shapes, all warp counts and both forms of the kernel (list for
+    """Eighty random (G, m, k, T) shapes, all warp counts and both forms of the kernel (list for
     k <= 56, dense above), some with duplicated columns or an all-zero sketch."""
     rs = np.random.default_rng(7)
     excused = total = 0
-    for trial in range(40):
+    for trial in range(80):
         G = int(rs.integers(2, 129)); m = int(rs.integers(2, 65)); k = int(rs.integers(1, G + 1)); T = int(rs.integers(0, 31))
         if trial % 5 == 0 and G >= 57:
             k = int(rs.integers(57, G + 1))
