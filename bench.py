@@ -53,6 +53,7 @@ def parse_args():
                     choices=["l2_7b_b1", "l2_7b_b64", "l3_8b_stack", "tiny_f32", "l2_13b_prompt"])
     ap.add_argument("--k", type=int, default=0, help="active groups (prompt workload sweep: 11 / 27 / 54)")
     ap.add_argument("--layers", type=int, default=0, help="distinct layers rotated through (0 = auto)")
+    ap.add_argument("--batch", type=int, default=0, help="decode batch override (regime sweeps; 0 = the workload's own)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     return ap.parse_args()
 
@@ -146,6 +147,8 @@ def run_ours(args):
     cfg = W.CONFIGS[args.workload]
     if args.k:
         cfg = cfg.with_(k=args.k)
+    if args.batch:
+        cfg = cfg.with_(B=args.batch)
     if cfg.prompt:
         return run_prompt(args, cfg, rank, world, local, dev)
     wbytes_layer = 3 * cfg.d_ff * cfg.d * (2 if cfg.w_dtype == "bf16" else 4)
@@ -272,7 +275,9 @@ def run_ours(args):
     ab = algorithmic_bytes(cfg, union)
     peak, _, peak_kind = peaks()
     exec_ms = stage_ms[2] + stage_ms[4]   # gather kernel, or gate/up + down GEMMs on the tensor-core path
-    mma = cfg.B >= 16 and cfg.w_dtype == "bf16" and cfg.group == 128
+    import math
+    mma_min = int(os.environ.get("CS_MMA_MIN_TOKENS", max(2, min(16, math.ceil(1.15 * cfg.G / cfg.k)))))
+    mma = cfg.B >= mma_min and cfg.w_dtype == "bf16" and cfg.group == 128
     # the dominant kernel reads the active weights and the hidden state, writes its partial sums
     kernel_bytes = ab["weights"] + cfg.B * cfg.d * 4 * 2
     achieved = kernel_bytes / (exec_ms * 1e-3) / 1e9 if exec_ms > 0 else None

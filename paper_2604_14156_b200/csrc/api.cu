@@ -1,6 +1,7 @@
 // The C boundary: plan life cycle, host-side validation and dispatch.  See include/cs.h.
 #include <math.h>
 #include <stdio.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include <new>
@@ -64,6 +65,14 @@ cs_status cs_plan_create(const cs_config *cfg, cs_plan **out) {
     alloc((void **)&p->colsum, (size_t)p->mean_row_blocks * cfg->d * sizeof(float));
     alloc((void **)&p->status, sizeof(DeviceStatus));
     p->mma_ok = cfg->w_dtype == CS_BF16 && cfg->group == 128 && cfg->d % 256 == 0;
+    // The gather path streams B * k groups, the tensor-core path every group once: it takes over where
+    // the first exceeds the second by the ~15 % the GEMM path costs extra (measured crossover between
+    // 4 and 5 tokens at G / k = 3.9; profiles/regime_sweep_l2_7b.md).
+    p->mma_min_tokens = max(2, min(kMmaMinTokens, (int)ceilf(1.15f * (float)p->G / (float)cfg->k)));
+    if (const char *ev = getenv("CS_MMA_MIN_TOKENS")) {   // regime sweeps: where the tensor-core path takes over
+        const int v = atoi(ev);
+        if (v >= 1 && v <= 129) p->mma_min_tokens = v;
+    }
     alloc((void **)&p->mask, nt * 4 * sizeof(uint32_t));
     alloc((void **)&p->gmask, (size_t)kMaxG * 4 * sizeof(uint32_t));
     alloc((void **)&p->counts, (size_t)kMaxG * sizeof(int32_t));
@@ -136,7 +145,7 @@ static cs_status check_weights(const cs_layer *L) {
 }
 
 extern "C++" {
-static bool use_decode_mma(const cs_plan *plan, int B) { return plan->mma_ok && B >= kMmaMinTokens && B <= 128; }
+static bool use_decode_mma(const cs_plan *plan, int B) { return plan->mma_ok && B >= plan->mma_min_tokens && B <= 128; }
 
 // Tensor-core decode path for 16..128 tokens.  The gate/up GEMM needs no supports (at these batch
 // sizes the union of the supports is, to within a group or two, every group), so it runs on the
@@ -172,7 +181,7 @@ static cs_status exec_decode_overlapped(cs_plan *plan, const cs_layer *layer, co
 // tokens) the token-tiled grouped GEMMs over the union list.
 static cs_status exec_dispatch(cs_plan *plan, const cs_layer *layer, const float *h, const int32_t *support,
                                int B, const float *residual, float *out, cudaStream_t st) {
-    if (!plan->mma_ok || B < kMmaMinTokens) return launch_ffn_gather(plan, layer, h, support, B, residual, out, st);
+    if (!plan->mma_ok || B < plan->mma_min_tokens) return launch_ffn_gather(plan, layer, h, support, B, residual, out, st);
     if (use_decode_mma(plan, B))
         return exec_decode_overlapped(plan, layer, h, B, residual, out, st,
                                       [&](cudaStream_t side) { return launch_bucket(plan, support, B, side); });

@@ -16,7 +16,8 @@ constexpr int kGatherThreads = 512;
 constexpr int kGatherMaxRows = 32;   // channel rows one gather CTA owns at most
 constexpr int kGatherMaxTokens = 16; // tokens per gather launch (scratch for partial sums)
 constexpr int kReduceGroups = 32;    // partial-sum groups of the deterministic cross-CTA reduction
-constexpr int kMmaMinTokens = 16;    // decode batches at least this large run on the tensor cores
+constexpr int kMmaMinTokens = 16;    // decode batches at least this large always run on the tensor cores; a plan
+                                     // lowers the bound by its G / k (CS_MMA_MIN_TOKENS overrides it, for sweeps)
 
 // Device status word values mirror cs_status (0 = ok).
 struct DeviceStatus {
@@ -53,6 +54,7 @@ struct cs_plan {
     void *act;           // [2][max_tokens, d_ff] bf16 SwiGLU activations over the group list (value, remainder)
     float *mma_partial;  // [slices, padded tokens, d] f32 partial down projections
     int mma_ok;          // shape qualifies for the tensor-core path
+    int mma_min_tokens;  // smallest decode batch that takes it
     int mma_slices;      // most list slices the down GEMM is split into
     int last_slices;
     float *x_host_in;  // [max_tokens, d] staging for the host-buffer entry point
@@ -132,7 +134,7 @@ cs_status launch_prompt_mean(cs_plan *plan, const void *H, int n, float *hbar, c
 // kernel launched the ordinary way (pdl = false).  Only the small-batch chain uses it: its kernels are
 // a few microseconds long and launch latency matters; with the large tensor-core kernels early-resident
 // dependents measurably slowed the step down.
-inline bool pdl_for(const cs_plan *plan, int B) { return !(plan->mma_ok && B >= kMmaMinTokens); }
+inline bool pdl_for(const cs_plan *plan, int B) { return !(plan->mma_ok && B >= plan->mma_min_tokens); }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
