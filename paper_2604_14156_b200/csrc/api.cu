@@ -67,7 +67,7 @@ cs_status cs_plan_create(const cs_config *cfg, cs_plan **out) {
     p->mma_ok = cfg->w_dtype == CS_BF16 && cfg->group == 128 && cfg->d % 256 == 0;
     // The gather path streams B * k groups, the tensor-core path every group once: it takes over where
     // the first exceeds the second by the ~15 % the GEMM path costs extra (measured crossover between
-    // 4 and 5 tokens at G / k = 3.9; profiles/regime_sweep_l2_7b.md).
+    // 4 and 5 tokens at G / k = 3.9).
     p->mma_min_tokens = max(2, min(kMmaMinTokens, (int)ceilf(1.15f * (float)p->G / (float)cfg->k)));
     if (const char *ev = getenv("CS_MMA_MIN_TOKENS")) {   // regime sweeps: where the tensor-core path takes over
         const int v = atoi(ev);
