@@ -550,9 +550,25 @@ ffn_gateup_swap_kernel(const __grid_constant__ CUtensorMap tm_g, const __grid_co
 
     if (warp == 0) {
         if (lane == 0) {
-            for (int kb = 0; kb < kblocks; ++kb) {
+            // Weights are parameters: the first ring of weight tiles is requested before the wait for the
+            // kernel that produces the token tiles (programmatic dependent launch), so the stream from
+            // HBM starts while that kernel is still running.
+            const int pre = min(stages, kblocks);
+            for (int kb = 0; kb < pre; ++kb) {
+                uint8_t *st = base + (size_t)kb * stage_bytes;
+                mbar_expect_tx(&bars->full[kb], stage_bytes);
+                tma_load_2d(st, &tm_g, kb * BK, g * 128, &bars->full[kb]);
+                tma_load_2d(st + kABytes, &tm_u, kb * BK, g * 128, &bars->full[kb]);
+            }
+            pdl_wait();
+            for (int kb = 0; kb < pre; ++kb) {
+                uint8_t *st = base + (size_t)kb * stage_bytes;
+                tma_load_2d(st + 2 * kABytes, &tm_x, kb * BK, 0, &bars->full[kb]);
+                if (SPLIT) tma_load_2d(st + 2 * kABytes + xbytes, &tm_x_lo, kb * BK, 0, &bars->full[kb]);
+            }
+            for (int kb = pre; kb < kblocks; ++kb) {
                 const int s = kb % stages;
-                if (kb >= stages && !mbar_wait(&bars->empty[s], ((kb / stages) - 1) & 1, bars, status)) break;
+                if (!mbar_wait(&bars->empty[s], ((kb / stages) - 1) & 1, bars, status)) break;
                 uint8_t *st = base + (size_t)s * stage_bytes;
                 mbar_expect_tx(&bars->full[s], stage_bytes);
                 tma_load_2d(st, &tm_g, kb * BK, g * 128, &bars->full[s]);
@@ -587,6 +603,7 @@ ffn_gateup_swap_kernel(const __grid_constant__ CUtensorMap tm_g, const __grid_co
         }
     } else {
         const int q = warp & 3, ch = q * 32 + lane;
+        pdl_wait();   // nothing is stored before the kernels before this one are complete
         if (mbar_wait(&bars->acc_ready, 0, bars, status)) {
             tc_fence_after();
             const uint32_t tbase = bars->tmem_base + ((uint32_t)(q * 32) << 16);
@@ -668,21 +685,34 @@ ffn_down_swap_kernel(const __grid_constant__ CUtensorMap tm_wd, const __grid_con
 
     if (warp == 0) {
         if (lane == 0) {
-            for (int kb = 0; kb < kblocks; ++kb) {
-                const int s = kb % stages;
-                if (kb >= stages && !mbar_wait(&bars->empty[s], ((kb / stages) - 1) & 1, bars, status)) break;
-                const int gi = gi0 + (kb >> 1), half = kb & 1;
-                const int wrow = glist[gi] * 128 + half * BK;
-                const int arow = (act_by_group ? glist[gi] : gi) * 128 + half * BK;
+            auto load_w = [&](int kb, int s) {   // weight tile of column tile j / 2: two blocks of 64 columns
+                const int wrow = glist[gi0 + (kb >> 1)] * 128 + (kb & 1) * BK;
                 uint8_t *st = base + (size_t)s * stage_bytes;
-                mbar_expect_tx(&bars->full[s], stage_bytes);
 #pragma unroll
-                for (int j = 0; j < 2 * CPC; ++j)   // weight tile of column tile j / 2: two blocks of 64 columns
+                for (int j = 0; j < 2 * CPC; ++j)
                     tma_load_2d(st + j * (64 * BK * 2), &tm_wd, c0 + j * 64, wrow, &bars->full[s]);
+            };
+            auto load_act = [&](int kb, int s) {
+                const int gi = gi0 + (kb >> 1);
+                const int arow = (act_by_group ? glist[gi] : gi) * 128 + (kb & 1) * BK;
+                uint8_t *st = base + (size_t)s * stage_bytes;
                 for (int i = 0; i < nblk; ++i) {
                     tma_load_2d(st + CPC * kABytes + i * (64 * BK * 2), &tm_act, i * 64, arow, &bars->full[s]);
                     if (SPLIT) tma_load_2d(st + CPC * kABytes + bbytes + i * (64 * BK * 2), &tm_act_lo, i * 64, arow, &bars->full[s]);
                 }
+            };
+            // as in the gate/up kernel: the first ring of weight tiles goes out before the wait for the
+            // kernel that completes the activations (the group list was final before that kernel began)
+            const int pre = min(stages, kblocks);
+            for (int kb = 0; kb < pre; ++kb) { mbar_expect_tx(&bars->full[kb], stage_bytes); load_w(kb, kb); }
+            pdl_wait();
+            for (int kb = 0; kb < pre; ++kb) load_act(kb, kb);
+            for (int kb = pre; kb < kblocks; ++kb) {
+                const int s = kb % stages;
+                if (!mbar_wait(&bars->empty[s], ((kb / stages) - 1) & 1, bars, status)) break;
+                mbar_expect_tx(&bars->full[s], stage_bytes);
+                load_w(kb, s);
+                load_act(kb, s);
             }
         }
     } else if (warp == 1) {
@@ -709,6 +739,7 @@ ffn_down_swap_kernel(const __grid_constant__ CUtensorMap tm_wd, const __grid_con
         }
     } else {
         const int q = warp & 3;
+        pdl_wait();   // nothing is stored before the kernels before this one are complete
         if (kblocks == 0) {
             for (int ct = 0; ct < CPC; ++ct) {
                 float *dst = partial + (size_t)z * 128 * d + c0 + ct * 128 + q * 32 + lane;
@@ -750,6 +781,7 @@ ffn_down_swap_kernel(const __grid_constant__ CUtensorMap tm_wd, const __grid_con
 // and 8-token chunk, for the value and the remainder matrix.
 __global__ void mask_act_kernel(__nv_bfloat16 *__restrict__ actT, __nv_bfloat16 *__restrict__ actT_lo,
                                 const uint32_t *__restrict__ gmask, int rows, int N) {
+    pdl_launch_dependents();   // the down GEMM may start streaming its weights
     const int chunks = N / 8;
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= rows * chunks) return;
@@ -793,6 +825,7 @@ __global__ void reduce_slices_kernel(const float *__restrict__ partial, int Z, i
 // x = y_hi + y_lo with both parts bf16: y_hi = round(x), y_lo = round(x - y_hi).
 __global__ void split_bf16_kernel(const float *__restrict__ x, __nv_bfloat16 *__restrict__ y_hi,
                                   __nv_bfloat16 *__restrict__ y_lo, size_t n4) {
+    pdl_launch_dependents();   // the gate/up GEMM may start streaming its weights
     const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n4) return;
     const float4 v = reinterpret_cast<const float4 *>(x)[i];
@@ -814,6 +847,7 @@ __global__ void __launch_bounds__(kNormSplitThreads)
 norm_split_bf16_kernel(const float *__restrict__ x, const float *__restrict__ gamma, float eps, int d,
                        __nv_bfloat16 *__restrict__ y_hi, __nv_bfloat16 *__restrict__ y_lo) {
     __shared__ float red[kNormSplitThreads / 32];
+    pdl_launch_dependents();   // the gate/up GEMM may start streaming its weights
     const int t = blockIdx.x, tid = threadIdx.x;
     const float4 *xr = reinterpret_cast<const float4 *>(x + (size_t)t * d);
     const float4 *gr = reinterpret_cast<const float4 *>(gamma);
@@ -1085,9 +1119,10 @@ cs_status launch_decode_gateup(cs_plan *plan, const cs_layer *L, const void *X, 
     CUtensorMap tm[7];
     if (!decode_maps(plan, L, X, X_lo, B, N, tm)) return record_cuda(plan, cudaErrorInvalidValue, "cuTensorMapEncodeTiled");
     StageTimer timer(plan, CS_STAGE_EXEC, st);
-    ffn_gateup_swap_kernel<true><<<plan->G, kMmaThreads, kMmaSmem, st>>>(
-        tm[0], tm[1], tm[2], tm[3], masked ? plan->glist : nullptr, plan->nu, N, c.d,
-        masked ? plan->gmask : nullptr, actT, actT_lo, plan->status);
+    launch_pdl(true, ffn_gateup_swap_kernel<true>, dim3(plan->G), dim3(kMmaThreads), kMmaSmem, st,
+               tm[0], tm[1], tm[2], tm[3], masked ? (const int32_t *)plan->glist : (const int32_t *)nullptr,
+               (const int32_t *)plan->nu, N, c.d, masked ? (const uint32_t *)plan->gmask : (const uint32_t *)nullptr,
+               actT, actT_lo, plan->status);
     plan->launches++;
     CS_CUDA_TRY(plan, cudaGetLastError());
     return CS_OK;
@@ -1113,8 +1148,9 @@ cs_status launch_decode_down(cs_plan *plan, const cs_layer *L, int B, bool act_b
     const int Z = max(1, min(plan->sm_count / (c.d / 256), 8));   // two column tiles per CTA (d is a multiple of 256)
     {
         StageTimer timer(plan, CS_STAGE_EXEC2, st);
-        ffn_down_swap_kernel<true, 2><<<dim3(c.d / 256, Z), kMmaThreads, kMmaSmem, st>>>(
-            tm[4], tm[5], tm[6], plan->glist, plan->nu, N, B, c.d, act_by_group ? 1 : 0, plan->mma_partial, plan->status);
+        launch_pdl(true, ffn_down_swap_kernel<true, 2>, dim3(c.d / 256, Z), dim3(kMmaThreads), kMmaSmem, st,
+                   tm[4], tm[5], tm[6], (const int32_t *)plan->glist, (const int32_t *)plan->nu, N, B, c.d,
+                   act_by_group ? 1 : 0, plan->mma_partial, plan->status);
         plan->launches++;
         CS_CUDA_TRY(plan, cudaGetLastError());
     }
