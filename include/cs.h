@@ -97,6 +97,21 @@ cs_status cs_recover(cs_plan *plan, const float *Phi, float mu, const float *y, 
                      int32_t *support, float *z, float *resid, void *stream);
 
 /*
+ * Warm-started estimator (Sec. 5: the support may be updated incrementally from the previous
+ * decoding step; Sec. 8 lists a warm start from the previous token among the cheap solvers; Sec. 11,
+ * incremental recovery under slow support drift).  The same iteration as cs_recover, T times, but
+ * from the k-sparse iterate z_0 with z_0[support0[t, j]] = z0[t, j] and zero elsewhere, e.g. the
+ * previous token's result, so that fewer iterations than the plan's T are needed when the support
+ * drifts slowly.  T >= 1 is this call's iteration count (the plan's is not used).
+ *   support0 [B,k] int32 ascending, distinct, in [0,G) (checked on the device, CS_ERR_SUPPORT through
+ *   cs_last_device_status), z0 [B,k] f32; other arguments and outputs as cs_recover.  The outputs may
+ *   alias the warm-start inputs.
+ */
+cs_status cs_recover_warm(cs_plan *plan, const float *Phi, float mu, const float *y, int32_t B, int32_t T,
+                          const int32_t *support0, const float *z0, int32_t *support, float *z, float *resid,
+                          void *stream);
+
+/*
  * Actuator (Sec. 3, execution only on the support), per token t with support s_t:
  *   a[c]   = silu(W_gate[c,:] . h_t) * (W_up[c,:] . h_t)     for every channel c of a group in s_t
  *   out[t] = (residual ? residual[t] : 0) + sum_c a[c] * Wd_t[c, :]

@@ -62,6 +62,7 @@ def load_library():
     lib.cs_plan_destroy.argtypes = [vp]
     lib.cs_sketch.argtypes = [vp, vp, vp, i32, vp, vp]
     lib.cs_recover.argtypes = [vp, vp, f32, vp, i32, vp, vp, vp, vp]
+    lib.cs_recover_warm.argtypes = [vp, vp, f32, vp, i32, i32, vp, vp, vp, vp, vp, vp]
     lib.cs_ffn_exec.argtypes = [vp, ctypes.POINTER(_Layer), vp, vp, i32, vp, vp, vp]
     lib.cs_layer_step.argtypes = [vp, ctypes.POINTER(_Layer), vp, i32, vp, vp, vp, vp, vp]
     lib.cs_prompt_support.argtypes = [vp, vp, vp, f32, vp, i32, vp, vp, vp, vp]
@@ -82,7 +83,7 @@ def load_library():
     lib.cs_status_string.restype = ctypes.c_char_p
     for name in ("cs_plan_create", "cs_plan_destroy", "cs_sketch", "cs_recover", "cs_ffn_exec",
                  "cs_layer_step", "cs_prompt_support", "cs_ffn_exec_shared", "cs_last_device_status",
-                 "cs_layer_step_host", "cs_plan_enable_timing", "cs_plan_stage_times"):
+                 "cs_layer_step_host", "cs_plan_enable_timing", "cs_plan_stage_times", "cs_recover_warm"):
         getattr(lib, name).restype = ctypes.c_int
     _lib = lib
     return lib
@@ -200,6 +201,21 @@ def cs_recover(plan: Plan, Phi, mu: float, y, stream=None):
     plan.check(plan.lib.cs_recover(plan.handle, _ptr(Phi, torch.float32, "Phi", (plan.m, plan.G)), float(mu),
                                    _ptr(y, torch.float32, "y", (B, plan.m)), B, support.data_ptr(),
                                    z.data_ptr(), resid.data_ptr(), _stream(stream)), "cs_recover")
+    return support, z, resid
+
+
+def cs_recover_warm(plan: Plan, Phi, mu: float, y, T: int, support0, z0, stream=None):
+    """T iterations from the k-sparse iterate (support0, z0) instead of zero; returns (support, z, resid)."""
+    B = y.shape[0]
+    dev = y.device
+    support = torch.empty((B, plan.k), dtype=torch.int32, device=dev)
+    z = torch.empty((B, plan.k), dtype=torch.float32, device=dev)
+    resid = torch.empty((B,), dtype=torch.float32, device=dev)
+    plan.check(plan.lib.cs_recover_warm(plan.handle, _ptr(Phi, torch.float32, "Phi", (plan.m, plan.G)), float(mu),
+                                        _ptr(y, torch.float32, "y", (B, plan.m)), B, int(T),
+                                        _ptr(support0, torch.int32, "support0", (B, plan.k)),
+                                        _ptr(z0, torch.float32, "z0", (B, plan.k)), support.data_ptr(),
+                                        z.data_ptr(), resid.data_ptr(), _stream(stream)), "cs_recover_warm")
     return support, z, resid
 
 

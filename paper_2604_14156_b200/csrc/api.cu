@@ -138,6 +138,19 @@ cs_status cs_recover(cs_plan *plan, const float *Phi, float mu, const float *y, 
     return launch_recover(plan, Phi, mu, y, B, support, z, resid, false, static_cast<cudaStream_t>(stream));
 }
 
+cs_status cs_recover_warm(cs_plan *plan, const float *Phi, float mu, const float *y, int32_t B, int32_t T,
+                          const int32_t *support0, const float *z0, int32_t *support, float *z, float *resid,
+                          void *stream) {
+    if (plan == nullptr || Phi == nullptr || y == nullptr || support0 == nullptr || z0 == nullptr || support == nullptr)
+        return CS_ERR_NULL;
+    if (B <= 0 || B > plan->cfg.max_tokens || T < 1) return CS_ERR_SHAPE;
+    if (!isfinite(mu) || !(mu > 0.f)) return CS_ERR_NONFINITE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cs_status s = launch_check_support(plan, support0, B, st);
+    if (s != CS_OK) return s;
+    return launch_recover(plan, Phi, mu, y, B, support, z, resid, false, st, T, support0, z0);
+}
+
 static cs_status check_weights(const cs_layer *L) {
     if (L == nullptr || L->W_gate == nullptr || L->W_up == nullptr || L->Wd_t == nullptr) return CS_ERR_NULL;
     if (!aligned16(L->W_gate) || !aligned16(L->W_up) || !aligned16(L->Wd_t)) return CS_ERR_UNSUPPORTED;

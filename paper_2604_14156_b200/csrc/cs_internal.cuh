@@ -106,7 +106,8 @@ cs_status launch_sketch(cs_plan *plan, const float *S, const float *x, const flo
                         float *y, float *n_out, const float *Phi, float mu, cudaStream_t st);
 // gram_ready: plan->gram already holds this Phi's matrix (the sketch launch before formed it).
 cs_status launch_recover(cs_plan *plan, const float *Phi, float mu, const float *y, int B,
-                         int32_t *support, float *z, float *resid, bool gram_ready, cudaStream_t st);
+                         int32_t *support, float *z, float *resid, bool gram_ready, cudaStream_t st,
+                         int T = -1 /* the plan's */, const int32_t *sup0 = nullptr, const float *z0 = nullptr);
 cs_status launch_ffn_gather(cs_plan *plan, const cs_layer *layer, const float *h, const int32_t *support,
                             int B, const float *residual, float *out, cudaStream_t st);
 cs_status prepare_ffn_gather(cs_plan *plan);

@@ -51,7 +51,7 @@ template <int NW, int KC>
 __global__ void __launch_bounds__(32 * NW)
 recover_kernel(const float *__restrict__ Phi, const float *__restrict__ gram, float mu, const float *__restrict__ y,
                int m, int G, int k, int T, int32_t *__restrict__ support, float *__restrict__ z_out,
-               float *__restrict__ resid_out) {
+               float *__restrict__ resid_out, const int32_t *__restrict__ sup0, const float *__restrict__ z0) {
     constexpr int GP = 32 * NW;                    // padded number of entries = pitch of M
     constexpr int NV = KC > 0 ? KC * 8 : GP;       // length of the iterate as the mat-vec reads it
     constexpr int NR = KC > 0 ? KC * 8 : GP;       // matrix entries a thread keeps
@@ -95,15 +95,33 @@ recover_kernel(const float *__restrict__ Phi, const float *__restrict__ gram, fl
         }
     }
     for (int row = tid; row < m; row += GP) y_s[row] = ld_dep(y + (size_t)t * m + row);
-    // z_0 = 0 with the support the order assigns to an all-zero vector: indices 0..k-1
-    for (int i = tid; i < NV; i += GP) {
-        val_s[0][i] = 0.f; val_s[1][i] = 0.f;
-        idx_s[i] = i < k ? i : 0;
-    }
-    bool kept = g < k;
-    int slot = g;
-    float v = 0.f;
+    // z_0 = 0 with the support the order assigns to an all-zero vector (indices 0..k-1), or, warm
+    // started, the k-sparse iterate handed in (sup0 ascending and distinct, z0 its values).
+    __shared__ int slot_s[GP];                     // warm start: list slot of each entry, -1 outside
+    const bool warm = sup0 != nullptr;
+    slot_s[g] = -1;
+    for (int i = tid; i < NV; i += GP) { val_s[0][i] = 0.f; val_s[1][i] = 0.f; idx_s[i] = i < k ? i : 0; }
     __syncthreads();
+    if (warm) {
+        for (int j = tid; j < k; j += GP) {
+            const int e = ld_dep(sup0 + (size_t)t * k + j);
+            const float zv = ld_dep(z0 + (size_t)t * k + j);
+            if ((unsigned)e >= (unsigned)G) continue;   // reported by the support check that ran before
+            slot_s[e] = j;
+            if constexpr (KC > 0) { idx_s[j] = e; val_s[0][j] = zv; }
+            else val_s[0][e] = zv;
+        }
+    }
+    __syncthreads();
+    bool kept = warm ? slot_s[g] >= 0 : g < k;
+    int slot = warm ? max(slot_s[g], 0) : g;
+    float v = 0.f;
+    if constexpr (KC > 0) {
+        if (warm) {   // the entries that go with the warm list
+#pragma unroll
+            for (int j = 0; j < NR; ++j) mreg[j] = ld_dep(mcol + idx_s[j] * GP);
+        }
+    }
     // c_g = mu sum_i Phi[i,g] y_i
     float cg = 0.f;
     if (valid && early_phi) {
@@ -231,7 +249,8 @@ recover_kernel(const float *__restrict__ Phi, const float *__restrict__ gram, fl
     }
 }
 
-typedef void (*RecoverFn)(const float *, const float *, float, const float *, int, int, int, int, int32_t *, float *, float *);
+typedef void (*RecoverFn)(const float *, const float *, float, const float *, int, int, int, int, int32_t *, float *, float *,
+                          const int32_t *, const float *);
 static int recover_kc(int k) { return k <= 56 ? (k + 7) / 8 : 0; }
 template <int NW> static RecoverFn recover_fn_kc(int k) {
     switch (recover_kc(k)) {
@@ -254,7 +273,8 @@ static RecoverFn recover_fn(int G, int k) {
     }
 }
 cs_status launch_recover(cs_plan *plan, const float *Phi, float mu, const float *y, int B, int32_t *support,
-                         float *z, float *resid, bool gram_ready, cudaStream_t st) {
+                         float *z, float *resid, bool gram_ready, cudaStream_t st, int T, const int32_t *sup0,
+                         const float *z0) {
     const cs_config &c = plan->cfg;
     const int G = plan->G;
     StageTimer timer(plan, CS_STAGE_RECOVER, st);
@@ -264,7 +284,7 @@ cs_status launch_recover(cs_plan *plan, const float *Phi, float mu, const float 
         CS_CUDA_TRY(plan, cudaGetLastError());
     }
     launch_pdl(pdl_for(plan, B), recover_fn(G, c.k), dim3(B), dim3(gram_pitch(G)), 0, st, Phi,
-               (const float *)plan->gram, mu, y, c.m, G, c.k, c.T, support, z, resid);
+               (const float *)plan->gram, mu, y, c.m, G, c.k, T < 0 ? c.T : T, support, z, resid, sup0, z0);
     plan->launches++;
     CS_CUDA_TRY(plan, cudaGetLastError());
     return CS_OK;

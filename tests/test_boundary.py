@@ -19,7 +19,8 @@ def lib():
 def test_library_exports_every_declared_symbol(lib):
     names = cs.exported_symbols()
     assert {"cs_plan_create", "cs_plan_destroy", "cs_sketch", "cs_recover", "cs_ffn_exec", "cs_layer_step",
-            "cs_prompt_support", "cs_ffn_exec_shared", "cs_last_device_status", "cs_status_string"} <= set(names)
+            "cs_prompt_support", "cs_ffn_exec_shared", "cs_last_device_status", "cs_status_string",
+            "cs_recover_warm"} <= set(names)
     for n in names:
         assert getattr(lib, n) is not None
 
@@ -48,6 +49,7 @@ def test_null_arguments_are_reported(lib):
     assert lib.cs_plan_destroy(None) == 1
     assert lib.cs_sketch(None, None, None, 1, None, None) == 1
     assert lib.cs_recover(None, None, 1.0, None, 1, None, None, None, None) == 1
+    assert lib.cs_recover_warm(None, None, 1.0, None, 1, 1, None, None, None, None, None, None) == 1
     assert lib.cs_layer_step(None, None, None, 1, None, None, None, None, None) == 1
     assert lib.cs_launch_count(None) == 0
 

@@ -149,6 +149,82 @@ def test_recover_random_shapes():
     assert excused <= total // 20
 
 
+def test_recover_warm_matches_oracle():
+    """Warm start (Sec. 5, Sec. 8): T iterations from the previous token's k-sparse iterate, against
+    the oracle started from the same dense z_0.  Random shapes over both kernel forms, a drifted y,
+    warm starts that hold zeros, outputs written over the warm-start buffers."""
+    rs = np.random.default_rng(11)
+    excused = total = 0
+    for trial in range(40):
+        G = int(rs.integers(2, 129)); m = int(rs.integers(2, 65)); k = int(rs.integers(1, G + 1))
+        if trial % 4 == 0 and G >= 57:
+            k = int(rs.integers(57, G + 1))
+        T0 = int(rs.integers(0, 21)); T1 = int(rs.integers(1, 9))
+        B = 4
+        Phi = torch.tensor(rs.normal(0, m ** -0.5, (m, G)), dtype=torch.float32)
+        mu = W.spectral_step(Phi)
+        y0 = torch.tensor(rs.normal(size=(B, m)), dtype=torch.float32)
+        y1 = y0 + 0.2 * torch.tensor(rs.normal(size=(B, m)), dtype=torch.float32)
+        plan = cs.Plan(256, G * 64, 64, m, k, T0, torch.float32, B, 1e-5)
+        Pd = Phi.to(DEV)
+        sup0, z0, _ = cs.cs_recover(plan, Pd, mu, y0.to(DEV))
+        if trial % 3 == 0:   # an arbitrary k-sparse start instead: random ascending support, some zero values
+            sup0 = torch.tensor(np.stack([np.sort(rs.choice(G, k, replace=False)) for _ in range(B)]), dtype=torch.int32, device=DEV)
+            z0 = torch.tensor(rs.normal(size=(B, k)) * (rs.random((B, k)) > 0.3), dtype=torch.float32, device=DEV)
+        s0 = sup0.cpu().numpy().copy(); v0 = z0.cpu().numpy().copy()
+        sup, z, resid = cs.cs_recover_warm(plan, Pd, mu, y1.to(DEV), T1, sup0, z0)
+        assert plan.device_status() == 0
+        if trial % 5 == 0:   # in place: the outputs are the warm-start buffers
+            lib = plan.lib
+            r2 = torch.empty(B, dtype=torch.float32, device=DEV)
+            plan.check(lib.cs_recover_warm(plan.handle, Pd.data_ptr(), float(mu), y1.to(DEV).data_ptr(), B, T1, sup0.data_ptr(),
+                                           z0.data_ptr(), sup0.data_ptr(), z0.data_ptr(), r2.data_ptr(), None), "cs_recover_warm")
+            torch.cuda.synchronize()
+            assert torch.equal(sup0, sup) and torch.equal(z0, z) and torch.equal(r2, resid)
+        sup = sup.cpu().numpy(); z = z.cpu().numpy(); resid = resid.cpu().numpy()
+        for t in range(B):
+            dense = np.zeros(G); dense[s0[t]] = v0[t]
+            ref = oracle.iht(Phi, y1[t], k, T1, mu, z0=dense)
+            total += 1
+            if np.array_equal(sup[t], ref.support):
+                zr = ref.z[ref.support]
+                assert (rel(z[t], zr) <= Z_TOL) if zr.any() else not z[t].any(), (G, m, k, T1, t)
+                assert abs(resid[t] - ref.resid) <= 1e-4 * max(1.0, ref.resid), (G, m, k, T1, t)
+            else:
+                assert ref.min_gap <= GAP_TOL, (G, m, k, T1, t, ref.min_gap)
+                excused += 1
+        plan.close()
+    assert excused <= total // 20
+
+
+def test_recover_warm_needs_fewer_iterations():
+    """Sec. 11 (slow support drift): from the previous token's result, a few iterations reach the
+    support that a cold start needs the plan's T for, on the benchmark's recovery shape."""
+    cfg = W.CONFIGS["l2_7b_b64"]
+    L = _layer(cfg)
+    tk = W.make_tokens(cfg, L.A, B=8)
+    plan = make_plan(cfg, max_tokens=8)
+    y = cs.cs_sketch(plan, L.S, tk.h.to(DEV))
+    sup_c, z_c, _ = cs.cs_recover(plan, L.Phi, L.mu, y)
+    # the next token's sketch: a small drift of this one's
+    g = torch.Generator().manual_seed(3)
+    y2 = y + 0.02 * y.abs().mean() * torch.randn(y.shape, generator=g).to(DEV)
+    sup_cold, _, _ = cs.cs_recover(plan, L.Phi, L.mu, y2)
+    sup_w, z_w, res_w = cs.cs_recover_warm(plan, L.Phi, L.mu, y2, 4, sup_c, z_c)
+    Phi = L.Phi.cpu(); yc = y2.cpu()
+    s0 = sup_c.cpu().numpy(); v0 = z_c.cpu().numpy()
+    agree = 0
+    for t in range(8):
+        dense = np.zeros(cfg.G); dense[s0[t]] = v0[t]
+        ref = oracle.iht(Phi, yc[t], cfg.k, 4, L.mu, z0=dense)
+        if ref.min_gap > GAP_TOL:
+            assert np.array_equal(sup_w[t].cpu().numpy(), ref.support), t
+            assert rel(z_w[t].cpu().numpy(), ref.z[ref.support]) <= Z_TOL
+        agree += len(set(sup_w[t].tolist()) & set(sup_cold[t].tolist()))
+    assert agree >= 0.95 * 8 * cfg.k   # 4 warm iterations land on (nearly) the cold start's T-iteration support
+    plan.close()
+
+
 @pytest.mark.parametrize("name,B", [("tiny_f32", 4), ("l2_7b_b1", 1), ("l2_7b_b64", 3)])
 def test_ffn_exec_matches_oracle_on_given_supports(name, B):
     cfg = W.CONFIGS[name]
