@@ -421,9 +421,10 @@ def test_bucket_inverts_supports():
     assert offsets[0] == 0 and offsets[cfg.G] == cfg.B * cfg.k
 
 
-@pytest.mark.parametrize("B", [16, 64, 100, 128, 130])
+@pytest.mark.parametrize("B", [5, 8, 11, 16, 64, 100, 128, 130])
 def test_ffn_exec_tensor_path_matches_oracle(B):
-    """Decode batches of 16 tokens and more run as grouped GEMMs over the union of the supports."""
+    """Decode batches from the crossover batch (5 tokens at this shape) up run as grouped GEMMs over
+    the union of the supports."""
     cfg = W.CONFIGS["l2_7b_b64"].with_(B=B)
     L = _layer(cfg)
     Lc = L.to("cpu")
@@ -433,9 +434,19 @@ def test_ffn_exec_tensor_path_matches_oracle(B):
     res = rng.normal(cfg.seed, (79,), (B, cfg.d), dtype=torch.float32)
     out = cs.cs_ffn_exec(plan, lay, tk.h.to(DEV), tk.planted.to(DEV), residual=res.to(DEV)).cpu().numpy()
     assert plan.device_status() == 0
-    for t in sorted({0, 1, B // 2, B - 2, B - 1}):
+    for t in (range(B) if B <= 16 else sorted({0, 1, B // 2, B - 2, B - 1})):
         ref = oracle.ffn(Lc.W_gate, Lc.W_up, Lc.Wd_t, cfg.group, tk.h[t], tk.planted[t])
         assert rel(out[t] - res[t].numpy(), ref) <= OUT_TOL["bf16"], t
+
+
+@pytest.mark.parametrize("B", [4, 5, 9])
+def test_layer_step_around_the_crossover_batch(B):
+    """The fused step on both sides of the batch where the tensor-core path takes over."""
+    cfg = W.CONFIGS["l2_7b_b64"].with_(B=B)
+    L = _layer(cfg)
+    tk = W.make_tokens(cfg, L.A, B=B)
+    rep, _, _ = compare_layer_step(cfg, L, make_plan(cfg, max_tokens=B), tk.h)
+    print(B, rep)
 
 
 def test_ffn_exec_tensor_path_skips_unused_groups():
