@@ -35,7 +35,7 @@ UNIT = "tokens/s"
 # ncu captures summarised under profiles/, keyed by (workload, k).  An entry is removed when its
 # kernel changes and comes back with the next capture; a missing entry reports null.
 NCU_TRAFFIC = {
-    ("l2_7b_b1", 22): 69.24e6 + 1.66e6,                       # ffn_gather_kernel
+    ("l2_7b_b1", 22): 69.24e6 + 1.60e6,                       # ffn_gather_kernel
     ("l2_7b_b64", 22): 181.44e6 + 3.97e6 + 95.85e6 + 5.02e6,  # ffn_gateup_swap_kernel + ffn_down_swap_kernel
     ("l2_13b_prompt", 27): 206.63e6 + 10.98e6 + 62.58e6 + 4.42e6,  # ffn_gateup_mma_kernel + ffn_down_mma_kernel
 }
