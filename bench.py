@@ -36,8 +36,8 @@ UNIT = "tokens/s"
 # kernel changes and comes back with the next capture; a missing entry reports null.
 NCU_TRAFFIC = {
     ("l2_7b_b1", 22): 69.24e6 + 1.60e6,                       # ffn_gather_kernel
-    ("l2_7b_b64", 22): 181.44e6 + 3.97e6 + 95.85e6 + 5.02e6,  # ffn_gateup_swap_kernel + ffn_down_swap_kernel
-    ("l2_13b_prompt", 27): 206.63e6 + 10.98e6 + 62.58e6 + 4.42e6,  # ffn_gateup_mma_kernel + ffn_down_mma_kernel
+    ("l2_7b_b64", 22): 181.47e6 + 3.81e6 + 95.85e6 + 3.66e6,  # ffn_gateup_swap_kernel + ffn_down_swap_kernel
+    ("l2_13b_prompt", 27): 206.07e6 + 10.58e6 + 58.22e6 + 4.15e6,  # ffn_gateup_mma_kernel + ffn_down_wide_kernel
 }
 GRAPH_STEPS = 64          # steps captured per CUDA graph
 N_TOKEN_BATCHES = 16      # distinct input batches rotated through
@@ -298,7 +298,7 @@ def run_ours(args):
         "clocks": clocks.summary(),
         "roofline": {"bound": "hbm",
                      "kernel": ("ffn_gateup_swap_kernel + ffn_down_swap_kernel" if cfg.B <= 128 else
-                                "ffn_gateup_mma_kernel + ffn_down_mma_kernel") if mma else "ffn_gather_kernel",
+                                "ffn_gateup_mma_kernel + ffn_down_wide_kernel (ffn_down_mma_kernel where it needs fewer rounds)") if mma else "ffn_gather_kernel",
                      "achieved": achieved, "peak": peak,
                      "unit": "GB/s", "frac": (achieved / peak) if achieved else None, "peak_kind": peak_kind,
                      "frac_of_8tbs_nominal": (achieved / 8000.0) if achieved else None,
@@ -411,7 +411,7 @@ def run_prompt(args, cfg, rank, world, local, dev):
         "e2e": {"value": tokens / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": cfg.B * cfg.d * 2,
                 "d2h_bytes_per_step": cfg.B * cfg.d * 2},
         "gpu_launches": launches, "clocks": clocks.summary(),
-        "roofline": {"bound": "tensor", "kernel": "ffn_gateup_mma_kernel + ffn_down_mma_kernel", "achieved": achieved,
+        "roofline": {"bound": "tensor", "kernel": "ffn_gateup_mma_kernel + ffn_down_wide_kernel (ffn_down_mma_kernel where it needs fewer rounds)", "achieved": achieved,
                      "peak": tf_peak, "unit": "TFLOP/s", "frac": achieved / tf_peak, "peak_kind": kind + " (sustained)",
                      "flops_per_launch_pair": flops, "avg_pair_us": stage_ms[2] * 1e3,
                      "traffic": NCU_TRAFFIC.get((cfg.name, cfg.k))},
