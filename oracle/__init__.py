@@ -216,6 +216,35 @@ def prompt_support(S, Phi, H, k: int, T: int, mu: float):
     return ybar, IHTResult(z, sup, rh, gh[:T])
 
 
+class BudgetResult:
+    __slots__ = ("H", "x", "m")
+
+    def __init__(self, H, x, m):
+        self.H, self.x, self.m = H, x, m
+
+
+def uds_budget(logits, m_base: float, gamma: float, m_min: int, m_max: int) -> BudgetResult:
+    """Uncertainty-driven measurement budget (Sec. 8.1, "Uncertainty-Driven Adaptive Sensing").
+
+    Per row of ``logits`` [B, V]: p = softmax(logits), H = -sum_v p_v log p_v (natural logarithm,
+    0 log 0 = 0), x = m_base (1 + gamma H), m = clip(floor(x), m_min, m_max).  fp64 throughout; x is
+    returned so that a comparison can tell how far the floor was from flipping.
+    """
+    L = _f64(logits)
+    if L.ndim == 1:
+        L = L[None, :]
+    H = np.empty(L.shape[0]); x = np.empty(L.shape[0]); m = np.empty(L.shape[0], dtype=np.int32)
+    for t in range(L.shape[0]):
+        row = L[t]
+        p = np.exp(row - row.max())
+        p = p / p.sum()
+        nz = p > 0
+        H[t] = -(p[nz] * np.log(p[nz])).sum()
+        x[t] = m_base * (1.0 + gamma * H[t])
+        m[t] = int(min(max(np.floor(x[t]), m_min), m_max))
+    return BudgetResult(H, x, m)
+
+
 def brute_force_support(Phi, y, k: int):
     """Best k-subset by exhaustive least squares: argmin_{|S|=k} min_c ||y - Phi_S c||.
 

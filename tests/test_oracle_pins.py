@@ -381,3 +381,51 @@ def test_prompt_support_uses_the_mean_sketch(oracle):
     ref = oracle.iht(L.Phi, ybar, cfg.k, cfg.T, L.mu)
     np.testing.assert_array_equal(it.support, ref.support)
     np.testing.assert_array_equal(it.z, ref.z)
+
+
+# ------------------------------------------------------------------ uncertainty-driven budget
+def test_uds_entropy_closed_forms(oracle):
+    """Uniform over V: H = log V.  n1 entries at logit a and n2 at logit b: the two-level closed
+    form.  A constant added to every logit changes nothing.  One dominant logit: H -> 0."""
+    for V in (2, 17, 1000, 32000):
+        r = oracle.uds_budget(np.full((1, V), 3.25), 1.0, 1.0, 0, 10 ** 9)
+        assert r.H[0] == pytest.approx(math.log(V), rel=1e-13)
+    n1, n2, a, b = 5, 11, 1.7, -0.4
+    Z = n1 * math.exp(a) + n2 * math.exp(b)
+    p1, p2 = math.exp(a) / Z, math.exp(b) / Z
+    want = -(n1 * p1 * math.log(p1) + n2 * p2 * math.log(p2))
+    row = np.array([a] * n1 + [b] * n2)
+    perm = np.random.default_rng(0).permutation(n1 + n2)
+    r = oracle.uds_budget(row[perm][None, :], 1.0, 1.0, 0, 10 ** 9)
+    assert r.H[0] == pytest.approx(want, rel=1e-13)
+    r2 = oracle.uds_budget(row[perm][None, :] + 123.0, 1.0, 1.0, 0, 10 ** 9)
+    assert r2.H[0] == pytest.approx(want, rel=1e-12)
+    spike = np.zeros((1, 500)); spike[0, 77] = 800.0   # exp underflows for the rest: 0 log 0 = 0
+    assert oracle.uds_budget(spike, 1.0, 1.0, 0, 10 ** 9).H[0] == 0.0
+
+
+def test_uds_entropy_matches_python_loop(oracle):
+    rs = np.random.default_rng(5)
+    L = rs.normal(0, 2.0, (3, 40))
+    r = oracle.uds_budget(L, 8.0, 0.5, 4, 64)
+    for t in range(3):
+        Z = sum(math.exp(v) for v in L[t])
+        H = -sum(math.exp(v) / Z * math.log(math.exp(v) / Z) for v in L[t])
+        assert r.H[t] == pytest.approx(H, rel=1e-12)
+        assert r.m[t] == min(max(math.floor(8.0 * (1 + 0.5 * H)), 4), 64)
+
+
+def test_uds_budget_formula_and_clipping(oracle):
+    """m = clip(floor(m_base (1 + gamma H))): worked values with H = log 4 (uniform over 4)."""
+    L = np.zeros((1, 4))                       # H = log 4 = 1.386...
+    assert oracle.uds_budget(L, 32, 0.5, 16, 64).m[0] == 54      # 32 * 1.6931 = 54.18
+    assert oracle.uds_budget(L, 32, 0.5, 16, 48).m[0] == 48      # upper bound
+    assert oracle.uds_budget(L, 4, 0.5, 16, 48).m[0] == 16       # lower bound: 6.77 -> 16
+    assert oracle.uds_budget(L, 32, 0.0, 1, 64).m[0] == 32       # gamma = 0: the base budget
+    sure = np.zeros((1, 9)); sure[0, 2] = 900.0
+    assert oracle.uds_budget(sure, 32, 0.5, 1, 64).m[0] == 32    # H = 0: the base budget
+    # entropy grows with temperature, so the budget is monotone in it
+    rs = np.random.default_rng(1)
+    base = rs.normal(size=(1, 300))
+    ms = [oracle.uds_budget(base / T, 16, 1.0, 1, 10 ** 6).m[0] for T in (0.1, 0.5, 1.0, 2.0, 10.0)]
+    assert ms == sorted(ms) and ms[0] < ms[-1]
