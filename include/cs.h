@@ -112,6 +112,24 @@ cs_status cs_recover_warm(cs_plan *plan, const float *Phi, float mu, const float
                           void *stream);
 
 /*
+ * Uncertainty-driven sensing controller (Sec. 8.1): per token, the predictive entropy of the
+ * previous decoding step's distribution over the vocabulary and the measurement budget for the
+ * current step,
+ *     p = softmax(logits[t, :]),  H = -sum_v p_v log p_v  (natural logarithm, 0 log 0 = 0),
+ *     m_t = clip(floor(m_base * (1 + gamma * H)), m_min, m_max).
+ *   logits [B,V] f32 (entries of -inf count as p = 0)  ->  m_t [B] int32, H [B] f32 (H may be NULL).
+ * The entropy is accumulated in f32 and the floor taken in double precision from it; a row whose
+ * entropy is NaN (a NaN or +inf logit) gets m_max.  The budget selects how many rows of the
+ * measurement bank the next cs_sketch / cs_recover use: S [m_max,d] and Phi [m_max,G] are row-major,
+ * so their first m_t rows are the operands of a plan created with m = m_t (with the step mu of that
+ * row prefix); the caller reads m_t back with the sampled token and picks the plan.
+ * Uses the plan's scratch: order it on the stream of the plan's other calls.  1 <= m_min <= m_max,
+ * m_base > 0, gamma >= 0, B <= max_tokens (else CS_ERR_SHAPE / CS_ERR_NONFINITE).
+ */
+cs_status cs_uds_budget(cs_plan *plan, const float *logits, int32_t B, int32_t V, float m_base, float gamma,
+                        int32_t m_min, int32_t m_max, float *H, int32_t *m_t, void *stream);
+
+/*
  * Actuator (Sec. 3, execution only on the support), per token t with support s_t:
  *   a[c]   = silu(W_gate[c,:] . h_t) * (W_up[c,:] . h_t)     for every channel c of a group in s_t
  *   out[t] = (residual ? residual[t] : 0) + sum_c a[c] * Wd_t[c, :]

@@ -63,6 +63,7 @@ def load_library():
     lib.cs_sketch.argtypes = [vp, vp, vp, i32, vp, vp]
     lib.cs_recover.argtypes = [vp, vp, f32, vp, i32, vp, vp, vp, vp]
     lib.cs_recover_warm.argtypes = [vp, vp, f32, vp, i32, i32, vp, vp, vp, vp, vp, vp]
+    lib.cs_uds_budget.argtypes = [vp, vp, i32, i32, f32, f32, i32, i32, vp, vp, vp]
     lib.cs_ffn_exec.argtypes = [vp, ctypes.POINTER(_Layer), vp, vp, i32, vp, vp, vp]
     lib.cs_layer_step.argtypes = [vp, ctypes.POINTER(_Layer), vp, i32, vp, vp, vp, vp, vp]
     lib.cs_prompt_support.argtypes = [vp, vp, vp, f32, vp, i32, vp, vp, vp, vp]
@@ -83,7 +84,7 @@ def load_library():
     lib.cs_status_string.restype = ctypes.c_char_p
     for name in ("cs_plan_create", "cs_plan_destroy", "cs_sketch", "cs_recover", "cs_ffn_exec",
                  "cs_layer_step", "cs_prompt_support", "cs_ffn_exec_shared", "cs_last_device_status",
-                 "cs_layer_step_host", "cs_plan_enable_timing", "cs_plan_stage_times", "cs_recover_warm"):
+                 "cs_layer_step_host", "cs_plan_enable_timing", "cs_plan_stage_times", "cs_recover_warm", "cs_uds_budget"):
         getattr(lib, name).restype = ctypes.c_int
     _lib = lib
     return lib
@@ -217,6 +218,17 @@ def cs_recover_warm(plan: Plan, Phi, mu: float, y, T: int, support0, z0, stream=
                                         _ptr(z0, torch.float32, "z0", (B, plan.k)), support.data_ptr(),
                                         z.data_ptr(), resid.data_ptr(), _stream(stream)), "cs_recover_warm")
     return support, z, resid
+
+
+def cs_uds_budget(plan: Plan, logits, m_base: float, gamma: float, m_min: int, m_max: int, stream=None):
+    """Entropy of softmax(logits[t]) and the budget clip(floor(m_base (1 + gamma H)), m_min, m_max); returns (m_t, H)."""
+    B, V = logits.shape
+    H = torch.empty((B,), dtype=torch.float32, device=logits.device)
+    m_t = torch.empty((B,), dtype=torch.int32, device=logits.device)
+    plan.check(plan.lib.cs_uds_budget(plan.handle, _ptr(logits, torch.float32, "logits", (B, V)), B, V, float(m_base),
+                                      float(gamma), int(m_min), int(m_max), H.data_ptr(), m_t.data_ptr(),
+                                      _stream(stream)), "cs_uds_budget")
+    return m_t, H
 
 
 def cs_ffn_exec(plan: Plan, layer: Layer, h, support, residual=None, out=None, stream=None):

@@ -151,6 +151,14 @@ cs_status cs_recover_warm(cs_plan *plan, const float *Phi, float mu, const float
     return launch_recover(plan, Phi, mu, y, B, support, z, resid, false, st, T, support0, z0);
 }
 
+cs_status cs_uds_budget(cs_plan *plan, const float *logits, int32_t B, int32_t V, float m_base, float gamma,
+                        int32_t m_min, int32_t m_max, float *H, int32_t *m_t, void *stream) {
+    if (plan == nullptr || logits == nullptr || m_t == nullptr) return CS_ERR_NULL;
+    if (B <= 0 || B > plan->cfg.max_tokens || V <= 0 || m_min < 1 || m_max < m_min) return CS_ERR_SHAPE;
+    if (!isfinite(m_base) || !(m_base > 0.f) || !isfinite(gamma) || gamma < 0.f) return CS_ERR_NONFINITE;
+    return launch_uds_budget(plan, logits, B, V, m_base, gamma, m_min, m_max, H, m_t, static_cast<cudaStream_t>(stream));
+}
+
 static cs_status check_weights(const cs_layer *L) {
     if (L == nullptr || L->W_gate == nullptr || L->W_up == nullptr || L->Wd_t == nullptr) return CS_ERR_NULL;
     if (!aligned16(L->W_gate) || !aligned16(L->W_up) || !aligned16(L->Wd_t)) return CS_ERR_UNSUPPORTED;

@@ -496,3 +496,96 @@ def test_ffn_exec_shared_ragged_prompt_length():
     for t in (0, 127, 128, 255, 256, 332):
         ref = oracle.ffn(Lc.W_gate, Lc.W_up, Lc.Wd_t, cfg.group, tk.h[t].double().numpy(), sup.cpu().numpy())
         assert rel(out[t], ref) <= OUT_TOL["bf16"], t
+
+
+# ------------------------------------------------------------------ uncertainty-driven budget
+def _check_budget(m_gpu, H_gpu, ref, m_base, gamma):
+    H_gpu = H_gpu.cpu().numpy().astype(np.float64); m_gpu = m_gpu.cpu().numpy()
+    for t in range(len(ref.H)):
+        assert abs(H_gpu[t] - ref.H[t]) <= 2e-5 * max(1.0, ref.H[t]), (t, H_gpu[t], ref.H[t])
+        # the floor may differ only where f32 rounding of H can carry x across an integer
+        slack = m_base * gamma * 2e-5 * max(1.0, ref.H[t])
+        if abs(ref.x[t] - round(ref.x[t])) > slack:
+            assert m_gpu[t] == ref.m[t], (t, m_gpu[t], ref.m[t], ref.x[t])
+        else:
+            assert abs(int(m_gpu[t]) - int(ref.m[t])) <= 1
+
+
+@pytest.mark.parametrize("B,V", [(1, 128256), (5, 32000), (64, 32000), (3, 50257), (2, 7), (4, 4096), (1, 1)])
+def test_uds_budget_matches_oracle(B, V):
+    """Sec. 8.1: entropy of the previous step's distribution and the budget it sets, at vocabulary
+    sizes of the benchmark's model families, ragged sizes, and temperatures from peaked to flat."""
+    g = torch.Generator().manual_seed(100 + B + V)
+    logits = torch.randn((B, V), generator=g) * torch.logspace(-1, 1.3, B)[:, None] + 3.0
+    plan = cs.Plan(256, 1024, 64, 8, 4, 4, torch.float32, max(B, 1), 1e-5)
+    m_base, gamma, m_min, m_max = 16.0, 0.75, 8, 64
+    m_t, H = cs.cs_uds_budget(plan, logits.to(DEV), m_base, gamma, m_min, m_max)
+    _check_budget(m_t, H, oracle.uds_budget(logits, m_base, gamma, m_min, m_max), m_base, gamma)
+    plan.close()
+
+
+def test_uds_budget_special_rows():
+    """Uniform row (H = log V), one dominant logit (H = 0, m = m_base), masked entries (-inf),
+    an entirely masked row, a NaN row (m_max), clipping at both ends, H not requested."""
+    V = 10000
+    L = torch.zeros((7, V))
+    L[1, 123] = 500.0
+    L[2] = torch.randn(V, generator=torch.Generator().manual_seed(1)); L[2, ::3] = float("-inf")
+    L[3] = float("-inf")
+    L[4, 5] = float("nan")
+    L[5] = torch.randn(V, generator=torch.Generator().manual_seed(2)) * 0.01     # near uniform: clipped at m_max
+    L[6, 0] = 40.0                                                               # near certain: H ~ 0
+    plan = cs.Plan(256, 1024, 64, 8, 4, 4, torch.float32, 8, 1e-5)
+    m_t, H = cs.cs_uds_budget(plan, L.to(DEV), 32.0, 0.5, 16, 100)
+    m = m_t.cpu().numpy(); Hh = H.cpu().numpy()
+    assert abs(Hh[0] - np.log(V)) < 1e-4 and m[0] == min(100, int(np.floor(32 * (1 + 0.5 * np.log(V)))))
+    assert Hh[1] == 0.0 and m[1] == 32
+    ref = oracle.uds_budget(L[2:3], 32.0, 0.5, 16, 100)
+    assert abs(Hh[2] - ref.H[0]) < 1e-4 and m[2] == ref.m[0]
+    assert Hh[3] == 0.0 and m[3] == 32
+    assert np.isnan(Hh[4]) and m[4] == 100
+    assert m[5] == 100 and m[6] == 32
+    lib = plan.lib
+    m2 = torch.empty(7, dtype=torch.int32, device=DEV)
+    Ld = L.to(DEV)
+    plan.check(lib.cs_uds_budget(plan.handle, Ld.data_ptr(), 7, V, 2.0, 0.5, 16, 100, None, m2.data_ptr(), None), "cs_uds_budget")
+    torch.cuda.synchronize()
+    assert (m2.cpu().numpy()[[0, 1, 6]] == 16).all()                             # lower bound
+    for bad, code in [((0, V, 2.0, 0.5, 16, 100), 2), ((9, V, 2.0, 0.5, 16, 100), 2), ((7, V, 2.0, 0.5, 0, 100), 2),
+                      ((7, V, 2.0, 0.5, 17, 16), 2), ((7, V, 0.0, 0.5, 16, 100), 5), ((7, V, 2.0, -1.0, 16, 100), 5),
+                      ((7, V, float("nan"), 0.5, 16, 100), 5)]:
+        assert lib.cs_uds_budget(plan.handle, Ld.data_ptr(), bad[0], bad[1], bad[2], bad[3], bad[4], bad[5], None,
+                                 m2.data_ptr(), None) == code, bad
+    plan.close()
+
+
+def test_uds_budget_selects_a_row_prefix_of_the_measurement_bank():
+    """Sec. 8.1 (the sensing matrix varies in its row dimension): the first m_t rows of a bank
+    S [m_max, d], Phi [m_max, G] are the operands of a plan created with m = m_t."""
+    cfg = W.CONFIGS["tiny_f32"]
+    m_max = 24
+    big = cfg.with_(m=m_max)
+    L = _layer(big)
+    tk = W.make_tokens(big, L.A, B=3)
+    logits = torch.randn((3, 5000), generator=torch.Generator().manual_seed(9)) * torch.tensor([8.0, 2.0, 0.2])[:, None]
+    ctl = make_plan(big, max_tokens=3)
+    m_t, _ = cs.cs_uds_budget(ctl, logits.to(DEV), 6.0, 0.35, 4, m_max)
+    m_t = m_t.cpu().numpy()
+    assert list(m_t) == list(oracle.uds_budget(logits, 6.0, 0.35, 4, m_max).m) and len(set(m_t)) == 3
+    for t in range(3):
+        mt = int(m_t[t])
+        plan = make_plan(big.with_(m=mt), max_tokens=1)
+        S_t, Phi_t = L.S[:mt], L.Phi[:mt]                    # contiguous row prefixes of the bank
+        assert S_t.is_contiguous() and Phi_t.is_contiguous()
+        mu = W.spectral_step(Phi_t.cpu())
+        x = tk.h[t:t + 1]
+        y = cs.cs_sketch(plan, S_t, x.to(DEV))
+        sup, z, _ = cs.cs_recover(plan, Phi_t, mu, y)
+        yr = oracle.sketch(S_t.cpu(), x[0])
+        ref = oracle.iht(Phi_t.cpu(), yr, big.k, big.T, mu)
+        assert rel(y[0].cpu().numpy(), yr) <= 1e-5
+        if ref.min_gap > GAP_TOL:
+            assert np.array_equal(sup[0].cpu().numpy(), ref.support)
+            assert rel(z[0].cpu().numpy(), ref.z[ref.support]) <= Z_TOL
+        plan.close()
+    ctl.close()
