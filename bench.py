@@ -291,7 +291,11 @@ def run_ours(args):
                    "m": cfg.m, "k": cfg.k, "T": cfg.T, "batch": cfg.B, "weights": cfg.w_dtype,
                    "accumulate": "f32", "layers_rotated": n_layers, "token_batches_rotated": N_TOKEN_BATCHES,
                    "l2": f"inputs larger than L2: {n_layers} layers x {wbytes_layer / 1e6:.0f} MB rotated",
-                   "cuda_graph_steps": chunk, "parallelism": f"dp{world}" if world > 1 else "single"},
+                   "cuda_graph_steps": chunk, "parallelism": f"dp{world}" if world > 1 else "single",
+                   "e2e_path": ("cs_layer_step_host on pinned host buffers: x fetched over the bus by a staging kernel, "
+                                "result stored into the host buffer by the step's last kernel"
+                                if cfg.B * cfg.d * 4 <= 65536 and not mma else
+                                "cs_layer_step_host on pinned host buffers: copy-engine transfers around the step")},
         "e2e": {"value": tokens / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": cfg.B * cfg.d * 4,
                 "d2h_bytes_per_step": cfg.B * cfg.d * 4},
         "gpu_launches": int(round(launches_per_step * K)),

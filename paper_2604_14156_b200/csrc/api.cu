@@ -35,6 +35,27 @@ static bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 
 
 using namespace cs;
 
+// Device-visible address of page-locked host memory (unified addressing), or NULL for pageable memory.
+static void *device_alias(const void *host) {
+    cudaPointerAttributes a;
+    if (cudaPointerGetAttributes(&a, host) != cudaSuccess) { cudaGetLastError(); return nullptr; }
+    return a.type == cudaMemoryTypeHost ? a.devicePointer : nullptr;
+}
+
+constexpr size_t kZeroCopyBytes = 64 * 1024;
+
+// x (page-locked host memory) -> plan scratch.  The host buffer is an input of the step, so it is
+// requested before the programmatic-launch wait; the store waits, because the kernels of the
+// step before may still be reading the scratch copy.
+__global__ void __launch_bounds__(256) stage_in_kernel(const float4 *src, float4 *dst, int n4) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    cs::pdl_launch_dependents();
+    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (i < n4) v = __ldcv(src + i);   // not cached: the host rewrites the buffer between steps
+    cs::pdl_wait();
+    if (i < n4) dst[i] = v;
+}
+
 extern "C" {
 
 cs_status cs_plan_create(const cs_config *cfg, cs_plan **out) {
@@ -285,10 +306,30 @@ cs_status cs_layer_step_host(cs_plan *plan, const cs_layer *layer, const float *
     if (s != CS_OK) return s;
     if (layer->S == nullptr || layer->Phi == nullptr) return CS_ERR_NULL;
     if (!isfinite(layer->mu) || !(layer->mu > 0.f)) return CS_ERR_NONFINITE;
-    CS_CUDA_TRY(plan, cudaMemcpyAsync(plan->x_host_in, x_host, bytes, cudaMemcpyHostToDevice, st));
-    s = cs_layer_step(plan, layer, plan->x_host_in, B, plan->x_host_out, plan->sup_buf, nullptr, nullptr, stream);
-    if (s != CS_OK) return s;
-    CS_CUDA_TRY(plan, cudaMemcpyAsync(x_out_host, plan->x_host_out, bytes, cudaMemcpyDeviceToHost, st));
+    // A few tokens in page-locked memory: the copy engine's set-up costs more than the transfer, so a
+    // kernel of the launch chain fetches x over the bus and the last kernel of the step stores the
+    // result straight into the caller's buffer.  Anything else goes through the copy engine.
+    const float *x_alias = nullptr;
+    float *out_alias = nullptr;
+    if (bytes <= kZeroCopyBytes && pdl_for(plan, B)) {
+        x_alias = static_cast<const float *>(device_alias(x_host));
+        out_alias = static_cast<float *>(device_alias(x_out_host));
+        if (x_alias == nullptr || out_alias == nullptr || !aligned16(x_alias) || !aligned16(out_alias)) x_alias = nullptr;
+    }
+    if (x_alias != nullptr) {
+        const int n4 = (int)(bytes / 16);
+        launch_pdl(true, stage_in_kernel, dim3((n4 + 255) / 256), dim3(256), 0, st,
+                   reinterpret_cast<const float4 *>(x_alias), reinterpret_cast<float4 *>(plan->x_host_in), n4);
+        plan->launches++;
+        CS_CUDA_TRY(plan, cudaGetLastError());
+        s = cs_layer_step(plan, layer, plan->x_host_in, B, out_alias, plan->sup_buf, nullptr, nullptr, stream);
+        if (s != CS_OK) return s;
+    } else {
+        CS_CUDA_TRY(plan, cudaMemcpyAsync(plan->x_host_in, x_host, bytes, cudaMemcpyHostToDevice, st));
+        s = cs_layer_step(plan, layer, plan->x_host_in, B, plan->x_host_out, plan->sup_buf, nullptr, nullptr, stream);
+        if (s != CS_OK) return s;
+        CS_CUDA_TRY(plan, cudaMemcpyAsync(x_out_host, plan->x_host_out, bytes, cudaMemcpyDeviceToHost, st));
+    }
     if (support_host != nullptr)
         CS_CUDA_TRY(plan, cudaMemcpyAsync(support_host, plan->sup_buf, (size_t)B * plan->cfg.k * sizeof(int32_t),
                                           cudaMemcpyDeviceToHost, st));

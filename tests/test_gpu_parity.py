@@ -589,3 +589,50 @@ def test_uds_budget_selects_a_row_prefix_of_the_measurement_bank():
             assert rel(z[0].cpu().numpy(), ref.z[ref.support]) <= Z_TOL
         plan.close()
     ctl.close()
+
+
+# ------------------------------------------------------------------ host-buffer entry point
+@pytest.mark.parametrize("name,B,pinned", [("l2_7b_b1", 1, True), ("l2_7b_b1", 1, False), ("tiny_f32", 4, True),
+                                           ("l2_7b_b64", 3, True), ("l2_7b_b64", 9, True), ("l2_7b_b64", 9, False)])
+def test_layer_step_host_matches_device_entry(name, B, pinned):
+    """Host buffers in, host buffers out: page-locked small batches travel inside the step's own
+    kernels, everything else through the copy engine; both give the device entry's bits, also when
+    the host rewrites the input between calls and when the calls are replayed from a graph."""
+    cfg = W.CONFIGS[name].with_(B=B)
+    L = _layer(cfg)
+    plan = make_plan(cfg, max_tokens=B)
+    lay = device_layer(plan, L)
+    hx = torch.empty((B, cfg.d), dtype=torch.float32)
+    hout = torch.empty((B, cfg.d), dtype=torch.float32)
+    hsup = torch.empty((B, cfg.k), dtype=torch.int32)
+    if pinned:
+        hx, hout, hsup = hx.pin_memory(), hout.pin_memory(), hsup.pin_memory()
+    for batch in range(3):
+        tk = W.make_tokens(cfg, L.A, batch=batch, B=B)
+        hx.copy_(tk.h)
+        hout.fill_(float("nan"))
+        cs.cs_layer_step_host(plan, lay, hx, hout, hsup if batch != 1 else None)
+        torch.cuda.synchronize()
+        want, sup, _, _ = cs.cs_layer_step(plan, lay, tk.h.to(DEV))
+        assert plan.device_status() == 0
+        assert torch.equal(hout, want.cpu()), batch
+        if batch != 1:
+            assert torch.equal(hsup, sup.cpu())
+    if pinned:
+        stream = torch.cuda.Stream()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(stream):
+            cs.cs_layer_step_host(plan, lay, hx, hout)
+            stream.synchronize()
+            with torch.cuda.graph(g, stream=stream):
+                for _ in range(3):
+                    cs.cs_layer_step_host(plan, lay, hx, hout)
+        for batch in (4, 5):
+            tk = W.make_tokens(cfg, L.A, batch=batch, B=B)
+            hx.copy_(tk.h)                      # the replay must see what the host wrote
+            hout.fill_(float("nan"))
+            g.replay()
+            torch.cuda.synchronize()
+            want, _, _, _ = cs.cs_layer_step(plan, lay, tk.h.to(DEV))
+            assert torch.equal(hout, want.cpu()), batch
+    plan.close()
