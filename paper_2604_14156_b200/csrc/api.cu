@@ -189,8 +189,8 @@ static cs_status check_weights(const cs_layer *L) {
 extern "C++" {
 static bool use_decode_mma(const cs_plan *plan, int B) { return plan->mma_ok && B >= plan->mma_min_tokens && B <= 128; }
 
-// Tensor-core decode path for 16..128 tokens.  The gate/up GEMM needs no supports (at these batch
-// sizes the union of the supports is, to within a group or two, every group), so it runs on the
+// Tensor-core decode path from the crossover batch (mma_min_tokens) up to 128 tokens.  The gate/up
+// GEMM needs no supports (at these batch sizes the union of the supports is, to within a group or two, every group), so it runs on the
 // caller's stream while `side_work` -- sketch / recovery / bucketing -- runs on the plan's second
 // stream; the two join before the activations are masked and the down GEMM starts.
 // gamma != NULL: h is the un-normalised x and the operand split applies the RMSNorm itself.

@@ -1091,8 +1091,8 @@ cs_status launch_ffn_mma(cs_plan *plan, const cs_layer *L, const void *X, const 
 }
 
 
-// Decode batches of 16..128 tokens in three launches that the caller orders (the gate/up GEMM can
-// run while the supports are still being recovered on another stream):
+// Decode batches from the crossover batch up to 128 tokens in three launches that the caller orders
+// (the gate/up GEMM can run while the supports are still being recovered on another stream):
 //   launch_decode_gateup(masked = false)  every group of the layer, activations unmasked, stored at the
 //                                         group's own index;   (masked = true: union list + masks)
 //   launch_decode_mask                    zeroes the (group, token) pairs outside the supports
