@@ -593,7 +593,8 @@ def test_uds_budget_selects_a_row_prefix_of_the_measurement_bank():
 
 # ------------------------------------------------------------------ host-buffer entry point
 @pytest.mark.parametrize("name,B,pinned", [("l2_7b_b1", 1, True), ("l2_7b_b1", 1, False), ("tiny_f32", 4, True),
-                                           ("l2_7b_b64", 3, True), ("l2_7b_b64", 9, True), ("l2_7b_b64", 9, False)])
+                                           ("l2_7b_b64", 3, True), ("l2_7b_b64", 9, True), ("l2_7b_b64", 9, False),
+                                           ("l3_8b_stack", 2, True)])   # RMSNorm + residual stream
 def test_layer_step_host_matches_device_entry(name, B, pinned):
     """Host buffers in, host buffers out: page-locked small batches travel inside the step's own
     kernels, everything else through the copy engine; both give the device entry's bits, also when
