@@ -245,6 +245,15 @@ def uds_budget(logits, m_base: float, gamma: float, m_min: int, m_max: int) -> B
     return BudgetResult(H, x, m)
 
 
+def support_drift(prev, cur) -> np.ndarray:
+    """Support drift between consecutive decoding steps (Sec. 11): Delta_t = |S_t symmetric-difference
+    S_{t-1}| per row of the two [B, k] index lists, by Python sets."""
+    a = _i32(prev); b = _i32(cur)
+    if a.ndim == 1:
+        a, b = a[None, :], b[None, :]
+    return np.array([len(set(a[t].tolist()) ^ set(b[t].tolist())) for t in range(a.shape[0])], dtype=np.int32)
+
+
 def brute_force_support(Phi, y, k: int):
     """Best k-subset by exhaustive least squares: argmin_{|S|=k} min_c ||y - Phi_S c||.
 

@@ -429,3 +429,12 @@ def test_uds_budget_formula_and_clipping(oracle):
     base = rs.normal(size=(1, 300))
     ms = [oracle.uds_budget(base / T, 16, 1.0, 1, 10 ** 6).m[0] for T in (0.1, 0.5, 1.0, 2.0, 10.0)]
     assert ms == sorted(ms) and ms[0] < ms[-1]
+
+
+def test_support_drift_worked_values(oracle):
+    """Sec. 11: Delta_t = |S_t symmetric-difference S_{t-1}|.  Equal supports: 0; disjoint: 2k; one
+    group replaced: 2; counted by hand for a small case."""
+    prev = np.array([[0, 1, 2, 3], [0, 1, 2, 3], [0, 1, 2, 3], [1, 4, 6, 9]], dtype=np.int32)
+    cur = np.array([[0, 1, 2, 3], [4, 5, 6, 7], [0, 1, 2, 9], [0, 4, 5, 9]], dtype=np.int32)
+    assert oracle.support_drift(prev, cur).tolist() == [0, 8, 2, 4]
+    assert oracle.support_drift(cur, prev).tolist() == [0, 8, 2, 4]      # symmetric
