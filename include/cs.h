@@ -112,6 +112,18 @@ cs_status cs_recover_warm(cs_plan *plan, const float *Phi, float mu, const float
                           void *stream);
 
 /*
+ * Support drift between consecutive decoding steps (Sec. 11, incremental recovery):
+ *     drift[t] = |S_t symmetric-difference S_{t-1}|
+ * for the supports of the previous and the current step, the quantity a caller watches to decide
+ * how many iterations (cs_recover_warm) or measurements the next step gets.
+ *   support_prev, support_cur [B,k] int32, ascending and distinct as cs_recover returns them
+ *   (checked on the device, CS_ERR_SUPPORT through cs_last_device_status)  ->  drift [B] int32,
+ *   even, between 0 and 2k.
+ */
+cs_status cs_support_drift(cs_plan *plan, const int32_t *support_prev, const int32_t *support_cur, int32_t B,
+                           int32_t *drift, void *stream);
+
+/*
  * Uncertainty-driven sensing controller (Sec. 8.1): per token, the predictive entropy of the
  * previous decoding step's distribution over the vocabulary and the measurement budget for the
  * current step,

@@ -7,5 +7,5 @@ shared library is missing and calls fail on non-CUDA tensors.
 """
 from .binding import (  # noqa: F401
     CSError, Layer, Plan, cs_bucket, cs_ffn_exec, cs_ffn_exec_shared, cs_ffn_exec_static, cs_layer_step, cs_layer_step_host, cs_prompt_support,
-    cs_recover, cs_recover_warm, cs_sketch, cs_uds_budget, exported_symbols, library_path, load_library,
+    cs_recover, cs_recover_warm, cs_sketch, cs_support_drift, cs_uds_budget, exported_symbols, library_path, load_library,
 )

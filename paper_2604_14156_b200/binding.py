@@ -64,6 +64,7 @@ def load_library():
     lib.cs_recover.argtypes = [vp, vp, f32, vp, i32, vp, vp, vp, vp]
     lib.cs_recover_warm.argtypes = [vp, vp, f32, vp, i32, i32, vp, vp, vp, vp, vp, vp]
     lib.cs_uds_budget.argtypes = [vp, vp, i32, i32, f32, f32, i32, i32, vp, vp, vp]
+    lib.cs_support_drift.argtypes = [vp, vp, vp, i32, vp, vp]
     lib.cs_ffn_exec.argtypes = [vp, ctypes.POINTER(_Layer), vp, vp, i32, vp, vp, vp]
     lib.cs_layer_step.argtypes = [vp, ctypes.POINTER(_Layer), vp, i32, vp, vp, vp, vp, vp]
     lib.cs_prompt_support.argtypes = [vp, vp, vp, f32, vp, i32, vp, vp, vp, vp]
@@ -84,7 +85,8 @@ def load_library():
     lib.cs_status_string.restype = ctypes.c_char_p
     for name in ("cs_plan_create", "cs_plan_destroy", "cs_sketch", "cs_recover", "cs_ffn_exec",
                  "cs_layer_step", "cs_prompt_support", "cs_ffn_exec_shared", "cs_last_device_status",
-                 "cs_layer_step_host", "cs_plan_enable_timing", "cs_plan_stage_times", "cs_recover_warm", "cs_uds_budget"):
+                 "cs_layer_step_host", "cs_plan_enable_timing", "cs_plan_stage_times", "cs_recover_warm", "cs_uds_budget",
+                 "cs_support_drift"):
         getattr(lib, name).restype = ctypes.c_int
     _lib = lib
     return lib
@@ -218,6 +220,16 @@ def cs_recover_warm(plan: Plan, Phi, mu: float, y, T: int, support0, z0, stream=
                                         _ptr(z0, torch.float32, "z0", (B, plan.k)), support.data_ptr(),
                                         z.data_ptr(), resid.data_ptr(), _stream(stream)), "cs_recover_warm")
     return support, z, resid
+
+
+def cs_support_drift(plan: Plan, support_prev, support_cur, stream=None):
+    """|S_t symmetric-difference S_{t-1}| per token for two [B, k] int32 support lists."""
+    B = support_cur.shape[0]
+    drift = torch.empty((B,), dtype=torch.int32, device=support_cur.device)
+    plan.check(plan.lib.cs_support_drift(plan.handle, _ptr(support_prev, torch.int32, "support_prev", (B, plan.k)),
+                                         _ptr(support_cur, torch.int32, "support_cur", (B, plan.k)), B,
+                                         drift.data_ptr(), _stream(stream)), "cs_support_drift")
+    return drift
 
 
 def cs_uds_budget(plan: Plan, logits, m_base: float, gamma: float, m_min: int, m_max: int, stream=None):

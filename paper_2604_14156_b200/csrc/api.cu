@@ -172,6 +172,17 @@ cs_status cs_recover_warm(cs_plan *plan, const float *Phi, float mu, const float
     return launch_recover(plan, Phi, mu, y, B, support, z, resid, false, st, T, support0, z0);
 }
 
+cs_status cs_support_drift(cs_plan *plan, const int32_t *support_prev, const int32_t *support_cur, int32_t B,
+                           int32_t *drift, void *stream) {
+    if (plan == nullptr || support_prev == nullptr || support_cur == nullptr || drift == nullptr) return CS_ERR_NULL;
+    if (B <= 0 || B > plan->cfg.max_tokens) return CS_ERR_SHAPE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cs_status s = launch_check_support(plan, support_prev, B, st);
+    if (s == CS_OK) s = launch_check_support(plan, support_cur, B, st);
+    if (s != CS_OK) return s;
+    return launch_support_drift(plan, support_prev, support_cur, B, drift, st);
+}
+
 cs_status cs_uds_budget(cs_plan *plan, const float *logits, int32_t B, int32_t V, float m_base, float gamma,
                         int32_t m_min, int32_t m_max, float *H, int32_t *m_t, void *stream) {
     if (plan == nullptr || logits == nullptr || m_t == nullptr) return CS_ERR_NULL;

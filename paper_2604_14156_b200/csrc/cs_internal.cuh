@@ -111,6 +111,8 @@ cs_status launch_recover(cs_plan *plan, const float *Phi, float mu, const float 
 cs_status launch_ffn_gather(cs_plan *plan, const cs_layer *layer, const float *h, const int32_t *support,
                             int B, const float *residual, float *out, cudaStream_t st);
 cs_status prepare_ffn_gather(cs_plan *plan);
+cs_status launch_support_drift(cs_plan *plan, const int32_t *prev, const int32_t *cur, int B, int32_t *drift,
+                               cudaStream_t st);
 cs_status launch_uds_budget(cs_plan *plan, const float *logits, int B, int V, float m_base, float gamma,
                             int m_min, int m_max, float *H, int32_t *m_t, cudaStream_t st);
 cs_status launch_check_support(cs_plan *plan, const int32_t *support, int B, cudaStream_t st);

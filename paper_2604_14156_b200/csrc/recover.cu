@@ -290,4 +290,35 @@ cs_status launch_recover(cs_plan *plan, const float *Phi, float mu, const float 
     return CS_OK;
 }
 
+// Support drift between consecutive decoding steps (Sec. 11): Delta_t = |S_t symmetric-difference
+// S_{t-1}|.  Both rows are ascending and distinct, so entry j of the new row is looked up in the old
+// one by bisection; the rows have k entries each, so the symmetric difference is twice the misses.
+constexpr int kDriftThreads = kMaxG;
+__global__ void __launch_bounds__(kDriftThreads)
+support_drift_kernel(const int32_t *__restrict__ prev, const int32_t *__restrict__ cur, int k,
+                     int32_t *__restrict__ drift) {
+    const int t = blockIdx.x, j = threadIdx.x;
+    const int32_t *p = prev + (size_t)t * k;
+    int missing = 0;
+    if (j < k) {
+        const int e = cur[(size_t)t * k + j];
+        int lo = 0, hi = k;                       // first index whose entry is >= e
+        while (lo < hi) {
+            const int mid = (lo + hi) >> 1;
+            if (p[mid] < e) lo = mid + 1; else hi = mid;
+        }
+        missing = !(lo < k && p[lo] == e);
+    }
+    const int n = __syncthreads_count(missing);
+    if (j == 0) drift[t] = 2 * n;
+}
+
+cs_status launch_support_drift(cs_plan *plan, const int32_t *prev, const int32_t *cur, int B, int32_t *drift,
+                               cudaStream_t st) {
+    support_drift_kernel<<<B, kDriftThreads, 0, st>>>(prev, cur, plan->cfg.k, drift);
+    plan->launches++;
+    CS_CUDA_TRY(plan, cudaGetLastError());
+    return CS_OK;
+}
+
 }  // namespace cs

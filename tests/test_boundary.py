@@ -51,6 +51,7 @@ def test_null_arguments_are_reported(lib):
     assert lib.cs_recover(None, None, 1.0, None, 1, None, None, None, None) == 1
     assert lib.cs_recover_warm(None, None, 1.0, None, 1, 1, None, None, None, None, None, None) == 1
     assert lib.cs_uds_budget(None, None, 1, 8, 1.0, 1.0, 1, 2, None, None, None) == 1
+    assert lib.cs_support_drift(None, None, None, 1, None, None) == 1
     assert lib.cs_layer_step(None, None, None, 1, None, None, None, None, None) == 1
     assert lib.cs_launch_count(None) == 0
 

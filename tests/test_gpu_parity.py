@@ -637,3 +637,35 @@ def test_layer_step_host_matches_device_entry(name, B, pinned):
             want, _, _, _ = cs.cs_layer_step(plan, lay, tk.h.to(DEV))
             assert torch.equal(hout, want.cpu()), batch
     plan.close()
+
+
+def test_support_drift_matches_oracle():
+    """Sec. 11: |S_t symmetric-difference S_{t-1}| for random supports (k from 1 to G), identical and
+    disjoint rows, and for the supports of two consecutive recoveries."""
+    rs = np.random.default_rng(21)
+    for G, k in [(86, 22), (112, 28), (128, 128), (16, 1), (108, 54), (128, 64)]:
+        B = 9
+        plan = cs.Plan(256, G * 64, 64, 8, k, 4, torch.float32, B, 1e-5)
+        prev = np.stack([np.sort(rs.choice(G, k, replace=False)) for _ in range(B)]).astype(np.int32)
+        cur = np.stack([np.sort(rs.choice(G, k, replace=False)) for _ in range(B)]).astype(np.int32)
+        cur[0] = prev[0]
+        if 2 * k <= G:
+            cur[1] = np.sort(np.setdiff1d(np.arange(G), prev[1])[:k])
+        got = cs.cs_support_drift(plan, torch.tensor(prev, device=DEV), torch.tensor(cur, device=DEV)).cpu().numpy()
+        assert plan.device_status() == 0
+        assert got.tolist() == oracle.support_drift(prev, cur).tolist(), (G, k)
+        assert got[0] == 0 and (2 * k > G or got[1] == 2 * k)
+        plan.close()
+    cfg = W.CONFIGS["l2_7b_b64"]
+    L = _layer(cfg)
+    tk = W.make_tokens(cfg, L.A, B=8)
+    plan = make_plan(cfg, max_tokens=8)
+    y = cs.cs_sketch(plan, L.S, tk.h.to(DEV))
+    s0, z0, _ = cs.cs_recover(plan, L.Phi, L.mu, y)
+    s1, _, _ = cs.cs_recover_warm(plan, L.Phi, L.mu, y * 1.02 + 0.05 * y.roll(1, 1), 4, s0, z0)
+    got = cs.cs_support_drift(plan, s0, s1).cpu().numpy()
+    assert got.tolist() == oracle.support_drift(s0.cpu().numpy(), s1.cpu().numpy()).tolist()
+    bad = s1.clone(); bad[2, 0] = bad[2, 1]                    # not ascending: flagged, not a fault
+    cs.cs_support_drift(plan, s0, bad)
+    assert plan.device_status() == 4
+    plan.close()
