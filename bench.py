@@ -323,7 +323,7 @@ def run_ours(args):
                    "cuda_graph_steps": chunk, "parallelism": f"dp{world}" if world > 1 else "single",
                    "e2e_path": ("cs_layer_step_host on pinned host buffers: x fetched over the bus by a staging kernel, "
                                 "result stored into the host buffer by the step's last kernel"
-                                if cfg.B * cfg.d * 4 <= 65536 and not mma else
+                                if cfg.B * cfg.d * 4 <= (4 << 20 if mma else 64 << 10) else
                                 "cs_layer_step_host on pinned host buffers: copy-engine transfers around the step")},
         "e2e": {"value": tokens / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": cfg.B * cfg.d * 4,
                 "d2h_bytes_per_step": cfg.B * cfg.d * 4},

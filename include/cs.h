@@ -235,9 +235,10 @@ cs_status cs_ffn_exec_shared(cs_plan *plan, const cs_layer *layer, const void *H
  * x_host [B,d] f32 to plan scratch, runs the step, copies x_out [B,d] f32 (and, if not NULL,
  * the supports [B,k] int32) back, all enqueued on `stream`.  The host buffers must stay valid
  * until the stream has been synchronised.  Per step it moves 4*B*d bytes each way.  When both
- * buffers are page-locked, 16-byte aligned and at most 64 KB (the small-batch regime), the bytes
- * cross the bus inside the step's own kernels (a staging kernel loads x, the last kernel stores
- * x_out into the caller's buffer) instead of through the copy engine; otherwise by cudaMemcpyAsync.
+ * buffers are page-locked, 16-byte aligned and small (at most 64 KB in the small-batch regime,
+ * 4 MB on the tensor-core path), the bytes cross the bus inside the step's own kernels (a staging
+ * kernel loads x, the last kernel stores x_out into the caller's buffer) instead of through the
+ * copy engine; otherwise by cudaMemcpyAsync.
  */
 cs_status cs_layer_step_host(cs_plan *plan, const cs_layer *layer, const float *x_host, int32_t B,
                              float *x_out_host, int32_t *support_host, void *stream);

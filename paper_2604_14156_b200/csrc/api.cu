@@ -43,6 +43,7 @@ static void *device_alias(const void *host) {
 }
 
 constexpr size_t kZeroCopyBytes = 64 * 1024;
+constexpr size_t kZeroCopyBytesLarge = 4 * 1024 * 1024;
 
 // x (page-locked host memory) -> plan scratch.  The host buffer is an input of the step, so it is
 // requested before the programmatic-launch wait; the store waits, because the kernels of the
@@ -317,19 +318,20 @@ cs_status cs_layer_step_host(cs_plan *plan, const cs_layer *layer, const float *
     if (s != CS_OK) return s;
     if (layer->S == nullptr || layer->Phi == nullptr) return CS_ERR_NULL;
     if (!isfinite(layer->mu) || !(layer->mu > 0.f)) return CS_ERR_NONFINITE;
-    // A few tokens in page-locked memory: the copy engine's set-up costs more than the transfer, so a
-    // kernel of the launch chain fetches x over the bus and the last kernel of the step stores the
-    // result straight into the caller's buffer.  Anything else goes through the copy engine.
+    // Small transfers from and to page-locked memory: the copy engine's set-up costs as much as the
+    // transfer or more, so a kernel of the launch chain fetches x over the bus and the last kernel of
+    // the step stores the result straight into the caller's buffer.  Anything else goes through the
+    // copy engine.
     const float *x_alias = nullptr;
     float *out_alias = nullptr;
-    if (bytes <= kZeroCopyBytes && pdl_for(plan, B)) {
+    if (bytes <= (pdl_for(plan, B) ? kZeroCopyBytes : kZeroCopyBytesLarge)) {
         x_alias = static_cast<const float *>(device_alias(x_host));
         out_alias = static_cast<float *>(device_alias(x_out_host));
         if (x_alias == nullptr || out_alias == nullptr || !aligned16(x_alias) || !aligned16(out_alias)) x_alias = nullptr;
     }
     if (x_alias != nullptr) {
         const int n4 = (int)(bytes / 16);
-        launch_pdl(true, stage_in_kernel, dim3((n4 + 255) / 256), dim3(256), 0, st,
+        launch_pdl(pdl_for(plan, B), stage_in_kernel, dim3((n4 + 255) / 256), dim3(256), 0, st,
                    reinterpret_cast<const float4 *>(x_alias), reinterpret_cast<float4 *>(plan->x_host_in), n4);
         plan->launches++;
         CS_CUDA_TRY(plan, cudaGetLastError());
