@@ -51,6 +51,32 @@ class StepReport:
     max_y_err: float
 
 
+def recovery_matches(sup_t, z_t, resid_t, ref, Phi, y_t, where=()) -> bool:
+    """One token's recovery (numpy support / z / resid) against the oracle's IHTResult.
+
+    True: same support, z within Z_TOL, residual norm within 1e-4.  False: it differs and the oracle met a
+    near-tie at some iteration (relative gap between the k-th and (k+1)-th magnitude <= GAP_TOL), after
+    which either order is a valid run of the algorithm -- also when the two runs end on the same support,
+    since with k > m the iterate remembers which of two tied entries was kept.  The caller counts such a
+    token as excused; the library's result must then still be consistent with itself (ascending distinct
+    support, resid = ||y - Phi z|| of its own z).  Anything else fails the test."""
+    k = len(sup_t)
+    zr = ref.z[ref.support]
+    same = np.array_equal(sup_t, ref.support)
+    if same:
+        z_ok = (rel(z_t, zr) <= Z_TOL) if zr.any() else not z_t.any()
+        r_ok = abs(resid_t - ref.resid) <= 1e-4 * max(1.0, ref.resid)
+        if z_ok and r_ok:
+            return True
+    assert ref.min_gap <= GAP_TOL, (where, "differs from the oracle with margin", ref.min_gap, "same support" if same else "")
+    G = Phi.shape[1]
+    assert (np.diff(sup_t) > 0).all() and sup_t[0] >= 0 and sup_t[-1] < G, where
+    own = np.asarray(y_t, dtype=np.float64) - np.asarray(Phi, dtype=np.float64)[:, sup_t] @ z_t.astype(np.float64)
+    own = float(np.linalg.norm(own))
+    assert abs(resid_t - own) <= 1e-4 * max(1.0, own), (where, resid_t, own)
+    return False
+
+
 def compare_layer_step(cfg: W.Config, L_dev: W.Layer, plan: cs.Plan, x_cpu: torch.Tensor,
                        add_residual=None) -> tuple[StepReport, np.ndarray, torch.Tensor]:
     """Runs cs_layer_step and the oracle on x; asserts the tolerances; returns the report, the
@@ -73,9 +99,14 @@ def compare_layer_step(cfg: W.Config, L_dev: W.Layer, plan: cs.Plan, x_cpu: torc
         assert (np.diff(sup[t]) > 0).all() and sup[t][0] >= 0 and sup[t][-1] < cfg.G
         if np.array_equal(sup[t], ref.support[t]):
             ez = rel(z[t], ref.z[t])
-            assert ez <= Z_TOL, (t, ez)
-            rep.max_z_err = max(rep.max_z_err, ez)
-            assert abs(resid[t] - ref.resid[t]) <= 1e-4 * max(1.0, ref.resid[t])
+            rz = abs(resid[t] - ref.resid[t]) / max(1.0, ref.resid[t])
+            if ez > Z_TOL or rz > 1e-4:
+                # same final support reached through a near-tie at some iteration: z may differ
+                # (the output below depends on the support only and is still compared)
+                assert ref.min_gap[t] <= GAP_TOL, (t, ez, rz, ref.min_gap[t])
+                excused += 1
+            else:
+                rep.max_z_err = max(rep.max_z_err, ez)
             eo = rel(out[t], ref.x_out[t])
             assert eo <= tol, (t, eo)
             rep.max_out_err = max(rep.max_out_err, eo)
