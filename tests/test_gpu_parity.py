@@ -311,6 +311,29 @@ def test_layer_step_ragged_shapes(shape, w):
     print(shape, w, rep)
 
 
+def test_layer_step_random_shapes():
+    """Forty random layer shapes through the fused step: both group sizes, d from 64 to 5120, any m, k,
+    T, batches on both sides of the crossover and past 128 tokens, both weight types, with and
+    without RMSNorm + residual."""
+    rs = np.random.default_rng(3)
+    for trial in range(40):
+        group = int(rs.choice([64, 128]))
+        G = int(rs.integers(2, 60))
+        d = int(rs.choice([64, 128, 192, 256, 320, 512, 768, 1024, 2048, 4096, 5120]))
+        m = int(rs.integers(2, 65)); k = int(rs.integers(1, G + 1)); T = int(rs.integers(0, 12))
+        B = int(rs.choice([1, 2, 3, 4, 5, 7, 9, 17, 33, 70, 130]))
+        w = str(rs.choice(["f32", "bf16"]))
+        base = W.CONFIGS["l3_8b_stack"] if rs.integers(0, 2) else W.CONFIGS["l2_7b_b64"]
+        cfg = base.with_(n_layers=1, w_dtype=w, T=T, d=d, d_ff=group * G, group=group, m=m, k=k, B=B,
+                         index=100 + trial)
+        L = _layer(cfg)
+        tk = W.make_tokens(cfg, L.A)
+        plan = make_plan(cfg)
+        rep, _, _ = compare_layer_step(cfg, L, plan, tk.h)
+        assert rep.excused <= max(1, B // 16), (trial, rep)
+        plan.close()
+
+
 def test_layer_step_in_place_and_without_aux_outputs():
     cfg = W.CONFIGS["l3_8b_stack"].with_(n_layers=1, d=512, d_ff=2048, m=16, k=4, B=6)
     L = _layer(cfg)
