@@ -504,6 +504,28 @@ def test_ffn_exec_shared_ragged_prompt_length():
         assert rel(out[t], ref) <= OUT_TOL["bf16"], t
 
 
+def test_ffn_exec_shared_random_shapes():
+    """Twenty random prompt-level shapes: d with and without the 320-column tiling, prompt lengths
+    around the 128-token tile, any k of G groups; sampled tokens against the oracle."""
+    rs = np.random.default_rng(5)
+    for trial in range(20):
+        G = int(rs.integers(2, 40)); k = int(rs.integers(1, G + 1))
+        d = int(rs.choice([256, 512, 768, 1024, 1280, 2560, 4096, 5120]))
+        n = int(rs.choice([1, 5, 127, 128, 129, 300, 640, 1000]))
+        cfg = W.CONFIGS["l2_13b_prompt"].with_(k=k, B=n, d=d, d_ff=128 * G, m=16, index=200 + trial)
+        L = _layer(cfg)
+        Lc = L.to("cpu")
+        tk = W.make_tokens(cfg, L.A)
+        plan = make_plan(cfg)
+        sup = torch.tensor(np.sort(rs.choice(G, k, replace=False)), dtype=torch.int32, device=DEV)
+        out = cs.cs_ffn_exec_shared(plan, device_layer(plan, L), tk.h.to(DEV), sup).float().cpu().numpy()
+        assert plan.device_status() == 0
+        for t in sorted({0, n // 2, n - 1, min(n - 1, 127), min(n - 1, 128)}):
+            ref = oracle.ffn(Lc.W_gate, Lc.W_up, Lc.Wd_t, cfg.group, tk.h[t].double().numpy(), sup.cpu().numpy())
+            assert rel(out[t], ref) <= OUT_TOL["bf16"], (trial, G, k, d, n, t)
+        plan.close()
+
+
 # ------------------------------------------------------------------ uncertainty-driven budget
 def _check_budget(m_gpu, H_gpu, ref, m_base, gamma):
     H_gpu = H_gpu.cpu().numpy().astype(np.float64); m_gpu = m_gpu.cpu().numpy()
