@@ -38,7 +38,8 @@ typedef enum {
     CS_ERR_SHAPE = 2,       /* sizes inconsistent with the plan (B > max_tokens, n <= 0, ...) */
     CS_ERR_UNSUPPORTED = 3, /* valid request outside the supported shapes / dtypes */
     CS_ERR_SUPPORT = 4,     /* device check: a support row is not ascending, distinct and in [0,G) */
-    CS_ERR_NONFINITE = 5,   /* host check: mu or rms_eps is not finite / not positive */
+    CS_ERR_NONFINITE = 5,   /* host check: mu or rms_eps is not finite / not positive; device check: a
+                               recovery met a NaN or infinite iterate (its outputs are valid indices, NaN values) */
     CS_ERR_CUDA = 6,        /* a CUDA runtime call failed; see cs_last_cuda_error */
     CS_ERR_TIMEOUT = 7      /* device check: a bounded wait inside a kernel gave up */
 } cs_status;
@@ -182,9 +183,11 @@ cs_status cs_bucket(cs_plan *plan, const int32_t *support, int32_t B, int32_t *c
  * allocating routine.
  *
  * Same mathematics, arguments and layouts as cs_ffn_exec (gather path), with the shape taken from
- * `cfg` (d, d_ff, group, k, w_dtype are read; m, T, max_tokens, rms_eps are ignored).  Supports
- * are not validated on the device: pass supports that are ascending, distinct and in [0, G), such
- * as cs_recover writes.
+ * `cfg` (d, d_ff, group, k, w_dtype are read; m, T, max_tokens, rms_eps are ignored).  Pointers must
+ * be 16-byte aligned (CS_ERR_UNSUPPORTED otherwise, before anything is launched).  There is no
+ * status word without a plan, so supports are not reported on: pass supports that are ascending,
+ * distinct and in [0, G), such as cs_recover writes.  A group index outside [0, G) is never turned
+ * into an address; the channels of such an entry contribute zero.
  *
  * Limit: B * nx * d * 4 bytes must fit in the 8 MiB array, where nx >= ceil(k * group / 32) is the
  * number of CTAs a token's rows are split over; e.g. d = 4096, k * group = 2816 allows B <= 5.
@@ -192,7 +195,11 @@ cs_status cs_bucket(cs_plan *plan, const int32_t *support, int32_t B, int32_t *c
  *
  * The first call on each device looks up the array's device address and raises the kernels'
  * shared-memory limit; make that first call with the device current and before any stream
- * capture begins.  All calls share the one array, which simply keeps whatever the last call
+ * capture begins.  If it is also the process's first use of the library on that device, the CUDA
+ * runtime loads the library's device code at that point, which places the 8 MiB array and may
+ * synchronise the device: make that call during start-up, not inside a latency-critical section.
+ * A failed launch is reported as CS_ERR_CUDA; if the second of the call's two kernels fails to
+ * launch, the first is already enqueued and `out` is left unwritten.  All calls share the one array, which simply keeps whatever the last call
  * left there (every call overwrites all it later reads, so nothing has to be cleared).  Two calls
  * whose kernels can overlap on the GPU -- different streams, or different host threads on the
  * same device -- would race on it: keep calls to this entry point ordered on one stream per device.
@@ -242,6 +249,17 @@ cs_status cs_ffn_exec_shared(cs_plan *plan, const cs_layer *layer, const void *H
  */
 cs_status cs_layer_step_host(cs_plan *plan, const cs_layer *layer, const float *x_host, int32_t B,
                              float *x_out_host, int32_t *support_host, void *stream);
+
+/*
+ * Regime crossover (Sec. 7: which precompiled execution path a batch takes).  Decode batches of at
+ * least `tokens` tokens (and at most 128) run on the tensor cores, smaller ones as the gather GEMV.
+ * A plan starts at max(2, min(16, ceil(1.15 * G / k))), the point where streaming every group once
+ * moves fewer bytes than streaming k groups per token; 1 <= tokens <= 129 (129: never below 129
+ * tokens).  Only shapes the tensor-core path supports (bf16 weights, 128-channel groups, d a
+ * multiple of 256) are affected.  cs_plan_crossover returns the current value.
+ */
+cs_status cs_plan_set_crossover(cs_plan *plan, int32_t tokens);
+int32_t cs_plan_crossover(const cs_plan *plan);
 
 /*
  * Stage timing (the paper asks for sensing / recovery overhead to be reported apart from the

@@ -71,6 +71,10 @@ def load_library():
     lib.cs_ffn_exec_shared.argtypes = [vp, ctypes.POINTER(_Layer), vp, i32, vp, vp, vp]
     lib.cs_layer_step_host.argtypes = [vp, ctypes.POINTER(_Layer), vp, i32, vp, vp, vp]
     lib.cs_plan_enable_timing.argtypes = [vp, i32]
+    lib.cs_plan_set_crossover.argtypes = [vp, i32]
+    lib.cs_plan_set_crossover.restype = ctypes.c_int
+    lib.cs_plan_crossover.argtypes = [vp]
+    lib.cs_plan_crossover.restype = ctypes.c_int32
     lib.cs_plan_stage_times.argtypes = [vp, vp, ctypes.POINTER(f32 * 5)]
     lib.cs_ffn_exec_static.argtypes = [ctypes.POINTER(_Config), ctypes.POINTER(_Layer), vp, vp, i32, vp, vp, vp]
     lib.cs_ffn_exec_static.restype = ctypes.c_int
@@ -141,6 +145,14 @@ class Plan:
         self.check(self.lib.cs_last_device_status(self.handle, _stream(stream), ctypes.byref(code)),
                    "cs_last_device_status")
         return code.value
+
+    @property
+    def crossover(self) -> int:
+        """Smallest decode batch that runs on the tensor cores."""
+        return int(self.lib.cs_plan_crossover(self.handle))
+
+    def set_crossover(self, tokens: int):
+        self.check(self.lib.cs_plan_set_crossover(self.handle, int(tokens)), "cs_plan_set_crossover")
 
     def enable_timing(self, on: bool = True):
         self.check(self.lib.cs_plan_enable_timing(self.handle, int(on)), "cs_plan_enable_timing")

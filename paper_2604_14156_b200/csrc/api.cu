@@ -1,7 +1,6 @@
 // The C boundary: plan life cycle, host-side validation and dispatch.  See include/cs.h.
 #include <math.h>
 #include <stdio.h>
-#include <stdlib.h>
 #include <string.h>
 
 #include <new>
@@ -45,16 +44,20 @@ static void *device_alias(const void *host) {
 constexpr size_t kZeroCopyBytes = 64 * 1024;
 constexpr size_t kZeroCopyBytesLarge = 4 * 1024 * 1024;
 
-// x (page-locked host memory) -> plan scratch.  The host buffer is an input of the step, so it is
-// requested before the programmatic-launch wait; the store waits, because the kernels of the
-// step before may still be reading the scratch copy.
+// x (page-locked host memory) -> plan scratch.  Both the load and the store come after the
+// programmatic-launch wait: whatever ran before on the stream may have written the host buffer (a
+// previous step that stored its result there, when layers are chained through one buffer) and may
+// still be reading the scratch copy.
 __global__ void __launch_bounds__(256) stage_in_kernel(const float4 *src, float4 *dst, int n4) {
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     cs::pdl_launch_dependents();
-    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (i < n4) v = __ldcv(src + i);   // not cached: the host rewrites the buffer between steps
     cs::pdl_wait();
-    if (i < n4) dst[i] = v;
+    if (i < n4) {
+        float4 v;   // volatile and uncached: the host (or the step before) rewrites the buffer between steps
+        asm volatile("ld.volatile.global.v4.f32 {%0, %1, %2, %3}, [%4];"
+                     : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(src + i) : "memory");
+        dst[i] = v;
+    }
 }
 
 extern "C" {
@@ -79,8 +82,6 @@ cs_status cs_plan_create(const cs_config *cfg, cs_plan **out) {
     alloc((void **)&p->n_buf, nt * cfg->d * sizeof(float));
     alloc((void **)&p->y_buf, nt * cfg->m * sizeof(float));
     alloc((void **)&p->sup_buf, nt * cfg->k * sizeof(int32_t));
-    alloc((void **)&p->z_buf, nt * cfg->k * sizeof(float));
-    alloc((void **)&p->resid_buf, nt * sizeof(float));
     alloc((void **)&p->partial, (size_t)kGatherMaxTokens * p->nx_max * cfg->d * sizeof(float));
     alloc((void **)&p->gram, (size_t)kMaxG * kMaxG * sizeof(float));
     alloc((void **)&p->hbar, (size_t)cfg->d * sizeof(float));
@@ -91,10 +92,6 @@ cs_status cs_plan_create(const cs_config *cfg, cs_plan **out) {
     // the first exceeds the second by the ~15 % the GEMM path costs extra (measured crossover between
     // 4 and 5 tokens at G / k = 3.9).
     p->mma_min_tokens = max(2, min(kMmaMinTokens, (int)ceilf(1.15f * (float)p->G / (float)cfg->k)));
-    if (const char *ev = getenv("CS_MMA_MIN_TOKENS")) {   // regime sweeps: where the tensor-core path takes over
-        const int v = atoi(ev);
-        if (v >= 1 && v <= 129) p->mma_min_tokens = v;
-    }
     alloc((void **)&p->mask, nt * 4 * sizeof(uint32_t));
     alloc((void **)&p->gmask, (size_t)kMaxG * 4 * sizeof(uint32_t));
     alloc((void **)&p->counts, (size_t)kMaxG * sizeof(int32_t));
@@ -131,8 +128,8 @@ cs_status cs_plan_create(const cs_config *cfg, cs_plan **out) {
 
 cs_status cs_plan_destroy(cs_plan *p) {
     if (p == nullptr) return CS_ERR_NULL;
-    cudaFree(p->n_buf); cudaFree(p->y_buf); cudaFree(p->sup_buf); cudaFree(p->z_buf);
-    cudaFree(p->resid_buf); cudaFree(p->partial); cudaFree(p->gram); cudaFree(p->hbar); cudaFree(p->colsum);
+    cudaFree(p->n_buf); cudaFree(p->y_buf); cudaFree(p->sup_buf);
+    cudaFree(p->partial); cudaFree(p->gram); cudaFree(p->hbar); cudaFree(p->colsum);
     cudaFree(p->status); cudaFree(p->x_host_in); cudaFree(p->x_host_out);
     cudaFree(p->mask); cudaFree(p->gmask); cudaFree(p->counts); cudaFree(p->offsets); cudaFree(p->token_ids); cudaFree(p->glist);
     cudaFree(p->nu); cudaFree(p->x_bf16); cudaFree(p->act); cudaFree(p->mma_partial);
@@ -233,9 +230,16 @@ static cs_status exec_decode_overlapped(cs_plan *plan, const cs_layer *layer, co
 
 // Dispatch of the actuator by batch size: gather GEMV, tensor-core decode path, or (more than 128
 // tokens) the token-tiled grouped GEMMs over the union list.
+// check: the supports come from the caller and are validated on the device (inside the gather
+// kernel, or by a small kernel ahead of the tensor-core paths).
 static cs_status exec_dispatch(cs_plan *plan, const cs_layer *layer, const float *h, const int32_t *support,
-                               int B, const float *residual, float *out, cudaStream_t st) {
-    if (!plan->mma_ok || B < plan->mma_min_tokens) return launch_ffn_gather(plan, layer, h, support, B, residual, out, st);
+                               int B, const float *residual, float *out, bool check, cudaStream_t st) {
+    if (!plan->mma_ok || B < plan->mma_min_tokens)
+        return launch_ffn_gather(plan, layer, h, support, B, residual, out, check, st);
+    if (check) {
+        cs_status s = launch_check_support(plan, support, B, st);
+        if (s != CS_OK) return s;
+    }
     if (use_decode_mma(plan, B))
         return exec_decode_overlapped(plan, layer, h, B, residual, out, st,
                                       [&](cudaStream_t side) { return launch_bucket(plan, support, B, side); });
@@ -255,10 +259,7 @@ cs_status cs_ffn_exec(cs_plan *plan, const cs_layer *layer, const float *h, cons
     if (s != CS_OK) return s;
     if (B <= 0 || B > plan->cfg.max_tokens) return CS_ERR_SHAPE;
     if (!aligned16(h) || !aligned16(out) || (residual != nullptr && !aligned16(residual))) return CS_ERR_UNSUPPORTED;
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
-    s = launch_check_support(plan, support, B, st);
-    if (s != CS_OK) return s;
-    return exec_dispatch(plan, layer, h, support, B, residual, out, st);
+    return exec_dispatch(plan, layer, h, support, B, residual, out, true, static_cast<cudaStream_t>(stream));
 }
 
 cs_status cs_bucket(cs_plan *plan, const int32_t *support, int32_t B, int32_t *counts, int32_t *offsets,
@@ -301,10 +302,14 @@ cs_status cs_layer_step(cs_plan *plan, const cs_layer *layer, const float *x, in
     }
     s = launch_sketch(plan, layer->S, x, layer->rms_gamma, B, plan->y_buf, norm ? plan->n_buf : nullptr, layer->Phi, layer->mu, st);
     if (s != CS_OK) return s;
+    const bool gather = !plan->mma_ok || B < plan->mma_min_tokens;
+    if (gather && fused_step_ok(plan))   // recovery and gather FFN in one launch: the weight stream starts on the first iterate
+        return launch_recover_gather(plan, layer, n, plan->y_buf, B, layer->add_residual ? x : nullptr, x_out, support_out,
+                                     z_out, resid_out, st);
     s = launch_recover(plan, layer->Phi, layer->mu, plan->y_buf, B, sup, z_out, resid_out, true, st);
     if (s != CS_OK) return s;
-    // supports produced by cs_recover are valid by construction: no device check here
-    return exec_dispatch(plan, layer, n, sup, B, layer->add_residual ? x : nullptr, x_out, st);
+    // supports produced by the recovery are valid by construction: no device check here
+    return exec_dispatch(plan, layer, n, sup, B, layer->add_residual ? x : nullptr, x_out, false, st);
 }
 
 cs_status cs_layer_step_host(cs_plan *plan, const cs_layer *layer, const float *x_host, int32_t B,
@@ -335,11 +340,13 @@ cs_status cs_layer_step_host(cs_plan *plan, const cs_layer *layer, const float *
                    reinterpret_cast<const float4 *>(x_alias), reinterpret_cast<float4 *>(plan->x_host_in), n4);
         plan->launches++;
         CS_CUDA_TRY(plan, cudaGetLastError());
-        s = cs_layer_step(plan, layer, plan->x_host_in, B, out_alias, plan->sup_buf, nullptr, nullptr, stream);
+        s = cs_layer_step(plan, layer, plan->x_host_in, B, out_alias, support_host != nullptr ? plan->sup_buf : nullptr, nullptr,
+                          nullptr, stream);
         if (s != CS_OK) return s;
     } else {
         CS_CUDA_TRY(plan, cudaMemcpyAsync(plan->x_host_in, x_host, bytes, cudaMemcpyHostToDevice, st));
-        s = cs_layer_step(plan, layer, plan->x_host_in, B, plan->x_host_out, plan->sup_buf, nullptr, nullptr, stream);
+        s = cs_layer_step(plan, layer, plan->x_host_in, B, plan->x_host_out, support_host != nullptr ? plan->sup_buf : nullptr,
+                          nullptr, nullptr, stream);
         if (s != CS_OK) return s;
         CS_CUDA_TRY(plan, cudaMemcpyAsync(x_out_host, plan->x_host_out, bytes, cudaMemcpyDeviceToHost, st));
     }
@@ -348,6 +355,15 @@ cs_status cs_layer_step_host(cs_plan *plan, const cs_layer *layer, const float *
                                           cudaMemcpyDeviceToHost, st));
     return CS_OK;
 }
+
+cs_status cs_plan_set_crossover(cs_plan *plan, int32_t tokens) {
+    if (plan == nullptr) return CS_ERR_NULL;
+    if (tokens < 1 || tokens > 129) return CS_ERR_SHAPE;
+    plan->mma_min_tokens = tokens;
+    return CS_OK;
+}
+
+int32_t cs_plan_crossover(const cs_plan *plan) { return plan != nullptr ? plan->mma_min_tokens : 0; }
 
 cs_status cs_plan_enable_timing(cs_plan *plan, int32_t on) {
     if (plan == nullptr) return CS_ERR_NULL;

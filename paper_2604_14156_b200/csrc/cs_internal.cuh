@@ -17,7 +17,7 @@ constexpr int kGatherMaxRows = 32;   // channel rows one gather CTA owns at most
 constexpr int kGatherMaxTokens = 16; // tokens per gather launch (scratch for partial sums)
 constexpr int kReduceGroups = 32;    // partial-sum groups of the deterministic cross-CTA reduction
 constexpr int kMmaMinTokens = 16;    // decode batches at least this large always run on the tensor cores; a plan
-                                     // lowers the bound by its G / k (CS_MMA_MIN_TOKENS overrides it, for sweeps)
+                                     // lowers the bound by its G / k (cs_plan_set_crossover overrides it)
 
 // Device status word values mirror cs_status (0 = ok).
 struct DeviceStatus {
@@ -35,8 +35,6 @@ struct cs_plan {
     float *n_buf;      // [max_tokens, d]  normalised FFN input
     float *y_buf;      // [max_tokens, m]
     int32_t *sup_buf;  // [max_tokens, k]
-    float *z_buf;      // [max_tokens, k]
-    float *resid_buf;  // [max_tokens]
     float *partial;    // [kGatherMaxTokens, nx_max, d] partial down-projections of the gather path
     float *gram;       // [G, pitch] I - mu Phi^T Phi of the layer being recovered, pitch = 32 ceil(G/32)
     float *hbar;       // [d] mean prompt hidden state
@@ -108,8 +106,14 @@ cs_status launch_sketch(cs_plan *plan, const float *S, const float *x, const flo
 cs_status launch_recover(cs_plan *plan, const float *Phi, float mu, const float *y, int B,
                          int32_t *support, float *z, float *resid, bool gram_ready, cudaStream_t st,
                          int T = -1 /* the plan's */, const int32_t *sup0 = nullptr, const float *z0 = nullptr);
+// check: validate the supports on the device (ascending, distinct, in range) inside the same launch
 cs_status launch_ffn_gather(cs_plan *plan, const cs_layer *layer, const float *h, const int32_t *support,
-                            int B, const float *residual, float *out, cudaStream_t st);
+                            int B, const float *residual, float *out, bool check, cudaStream_t st);
+// the small-batch step in one launch: recovery of y beside the gather FFN that starts on its first iterate
+bool fused_step_ok(const cs_plan *plan);
+cs_status launch_recover_gather(cs_plan *plan, const cs_layer *layer, const float *h, const float *y, int B,
+                                const float *residual, float *out, int32_t *support, float *z, float *resid,
+                                cudaStream_t st);
 cs_status prepare_ffn_gather(cs_plan *plan);
 cs_status launch_support_drift(cs_plan *plan, const int32_t *prev, const int32_t *cur, int B, int32_t *drift,
                                cudaStream_t st);

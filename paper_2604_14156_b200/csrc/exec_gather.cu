@@ -1,7 +1,8 @@
 // Actuator, small-batch regime: a gather GEMV that streams every active weight row exactly once.
 //
-// The k*b active channel rows of a token are split evenly over the CTAs of its grid row.  A CTA
-// owns a contiguous range of channel rows and does, for those rows only,
+// The k*b active channel rows of a token (row R = slot * b + channel, slot = position in the
+// token's support list) are dealt out to the CTAs of its grid row like cards: CTA x owns rows
+// x, x + nx, x + 2 nx, ...  For its rows a CTA does
 //     a[c]      = silu(W_gate[c,:] . h) * (W_up[c,:] . h)
 //     partial[:] = sum_c a[c] * Wd_t[c,:]
 // so gate, up and down rows of a channel are consumed by the same CTA and nothing but the
@@ -20,7 +21,21 @@
 //     its gate/up units, i.e. they are in flight while the activations are being folded.
 // The partial d-vectors are summed in a fixed order by reduce_partials_kernel (deterministic,
 // no atomics), which also adds the residual.
-#include "cs_internal.cuh"
+//
+// FUSED (cs_layer_step at small batches): the supports are not an input.  Four extra warps of every
+// CTA run the recovery of the CTA's token (recover_core.cuh; every CTA of a token repeats it, which
+// costs nothing that matters: a few KB from L2), and the 16 streaming warps start on the support of
+// the FIRST iteration while the other iterations run.  The recovery keeps its support as a table of
+// k stable slots (slot -> group) in shared memory; the streaming warps read the table when they
+// request a row and remember which group they requested.  The first iteration hands the slots out
+// by decreasing magnitude and rows are dealt to CTAs and requested in slot order, so the rows
+// requested first belong to the entries least likely to leave the support, and a slot that does
+// change costs every CTA at most one row (not one CTA all of its rows).  When the recovery has
+// finished, units whose remembered group is not the slot's final one are fetched and computed
+// again; the down phase only ever uses the final table.
+#include <type_traits>
+
+#include "recover_core.cuh"
 
 namespace cs {
 
@@ -35,6 +50,19 @@ constexpr int kUnitStages = kWarpRing / kUnitBytes;        // 3 units in flight 
 constexpr int kLaneSlots = kWarpRing / (32 * 16);          // 24 chunks per lane in the down phase
 constexpr int kMaxSegs = kMaxD * 4 / (kUnitChunks * 32 * 16);  // 16 (f32 rows of 8192)
 
+// Recovery side of the fused kernel: G <= 128 entries on four warps, list form with up to 32 slots.
+constexpr int kFusedNW = 4, kFusedKC = 4;
+constexpr int kFusedMaxK = 8 * kFusedKC;
+constexpr int kFusedThreads = kGatherThreads + 32 * kFusedNW;
+struct FusedArgs {
+    const float *Phi, *gram, *y;   // [m,G], [G,pitch], [B,m]
+    float mu;
+    int m, T, pitch;
+    int32_t *support;              // [B,k] ascending (may be NULL)
+    float *z, *resid;              // [B,k], [B] (may be NULL)
+};
+struct NoSmem {};
+
 __device__ __forceinline__ void cp_async16(void *smem_dst, const void *gmem_src) {
     const uint32_t s = static_cast<uint32_t>(__cvta_generic_to_shared(smem_dst));
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(s), "l"(gmem_src) : "memory");
@@ -46,11 +74,12 @@ template <int N> __device__ __forceinline__ void cp_async_wait() {
 
 // CPT = 16-byte chunks per thread and row in the down phase (row bytes / (512 * 16), rounded up).
 // FULL = every row is a whole number of units and of 512-chunk slices: no bounds checks inside.
-template <typename WT, int CPT, bool FULL>
-__global__ void __launch_bounds__(kGatherThreads, 1)
+// check: the CTAs with blockIdx.x == 0 also validate their token's support row (ascending, distinct).
+template <typename WT, int CPT, bool FULL, bool FUSED>
+__global__ void __launch_bounds__(FUSED ? kFusedThreads : kGatherThreads, 1)
 ffn_gather_kernel(const WT *__restrict__ Wg, const WT *__restrict__ Wu, const WT *__restrict__ Wdt,
-                  const float *__restrict__ h, const int32_t *__restrict__ support, int d, int b, int k,
-                  float *__restrict__ partial) {
+                  const float *__restrict__ h, const int32_t *__restrict__ support, int d, int lb, int k, int G,
+                  float *__restrict__ partial, DeviceStatus *status, int check, FusedArgs fa) {
     constexpr int E = Chunk<WT>::kElems;
     constexpr int DR = kLaneSlots / CPT;               // down rows in flight per thread
     constexpr int kSegElems = kUnitChunks * 32 * E;    // elements of one row segment
@@ -58,24 +87,65 @@ ffn_gather_kernel(const WT *__restrict__ Wg, const WT *__restrict__ Wu, const WT
     __shared__ float red[kGatherMaxRows][kMaxSegs][2];
     __shared__ float a_s[kGatherMaxRows];
     __shared__ int chan_s[kGatherMaxRows];
+    __shared__ int bad_s[kGatherMaxRows];   // row belongs to a group index outside [0, G): contributes nothing
+    __shared__ short ugrp_s[FUSED ? kGatherMaxRows : 1][FUSED ? kMaxSegs : 1];   // group each unit was requested for
+    __shared__ typename std::conditional<FUSED, RecoverSmem<kFusedNW, kFusedKC>, NoSmem>::type rs;
 
-    const int t = blockIdx.y, nx = gridDim.x;
-    const int rows_total = k * b;
-    const int r_begin = (int)(((long long)rows_total * blockIdx.x) / nx);
-    const int r_end = (int)(((long long)rows_total * (blockIdx.x + 1)) / nx);
-    const int nrows = r_end - r_begin;
+    const int t = blockIdx.y, nx = gridDim.x, bx = blockIdx.x;
+    const int b = 1 << lb;
+    const int rows_total = k << lb;
+    const int nrows = (rows_total - bx + nx - 1) / nx;     // rows bx, bx + nx, ...
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    auto cta_sync = [] {   // the streaming warps only
+        if constexpr (FUSED) bar_sync<1, kGatherThreads>(); else __syncthreads();
+    };
+    pdl_launch_dependents();
+    if constexpr (FUSED) {
+        if (tid >= kGatherThreads) {   // the recovery warps
+            const int g = tid - kGatherThreads;
+            float phc[32];
+            if (fa.m <= 32) recover_load_phi<kFusedNW>(fa.Phi, fa.m, G, g, phc);
+            pdl_wait();   // y and M come from the kernel before
+            const bool writer = bx == 0;   // every CTA of the token finds the same result; one writes it
+            recover_token<kFusedNW, kFusedKC, 4>(
+                rs, g, fa.Phi, fa.gram, fa.pitch, fa.mu, fa.y + (size_t)t * fa.m, fa.m, G, k, fa.T,
+                writer && fa.support != nullptr ? fa.support + (size_t)t * k : nullptr,
+                writer && fa.z != nullptr ? fa.z + (size_t)t * k : nullptr,
+                writer && fa.resid != nullptr ? fa.resid + t : nullptr, nullptr, nullptr, writer ? status : nullptr, phc,
+                [] { __threadfence_block(); bar_arrive<2, kFusedThreads>(); },   // the streaming warps may start
+                [] { __threadfence_block(); bar_arrive<3, kFusedThreads>(); });  // the table is final
+            return;
+        }
+    }
     const int chunks = d / E;                                       // chunks per row
     const int nseg = (chunks + kUnitChunks * 32 - 1) / (kUnitChunks * 32);
     const int nunits = nrows * nseg;
-    pdl_launch_dependents();
     pdl_wait();   // supports and activations come from the kernels before
 
-    if (tid < nrows) {
-        const int c = r_begin + tid;
-        chan_s[tid] = ld_dep(support + (size_t)t * k + c / b) * b + c % b;
+    if constexpr (!FUSED) {
+        if (tid < nrows) {
+            const int R = bx + nx * tid;
+            // A group index outside [0, G) must not become an address: the row is read from group 0
+            // instead, its activation is forced to zero, and the call's status word (if any) says so.
+            int g = ld_dep(support + (size_t)t * k + (R >> lb));
+            const bool bad = (unsigned)g >= (unsigned)G;
+            if (bad) {
+                g = 0;
+                if (status != nullptr) atomicCAS(&status->code, 0, (int)CS_ERR_SUPPORT);
+            }
+            bad_s[tid] = bad;
+            chan_s[tid] = (g << lb) + (R & (b - 1));
+        }
+        if (check && bx == 0 && status != nullptr && tid >= kGatherThreads - kMaxG && tid - (kGatherThreads - kMaxG) < k) {
+            // the last warps of the first CTA check the row: ascending, hence distinct (the range is checked above)
+            const int j = tid - (kGatherThreads - kMaxG);
+            if (j > 0 && ld_dep(support + (size_t)t * k + j) <= ld_dep(support + (size_t)t * k + j - 1))
+                atomicCAS(&status->code, 0, (int)CS_ERR_SUPPORT);
+        }
+        __syncthreads();
     }
-    __syncthreads();
+    volatile const int *table = nullptr;               // FUSED: the recovery's live slot table
+    if constexpr (FUSED) table = rs.idx;
 
     uint4 *wring = ring + (size_t)warp * (kWarpRing / 16) + lane;   // this lane's column of the warp ring
     // ---- gate / up: units u = warp, warp + 16, ... ; unit u = (row u / nseg, segment u % nseg).
@@ -90,25 +160,33 @@ ffn_gather_kernel(const WT *__restrict__ Wg, const WT *__restrict__ Wu, const WT
     const WT *wg_lane = Wg + lane * E, *wu_lane = Wu + lane * E;
     const float *h_lane = h + (size_t)t * d + lane * E;
 
-    auto issue_unit = [&](int stage) {
-        if (ci.u < nunits) {
-            const size_t off = (size_t)chan_s[ci.r] * d + (size_t)ci.seg * kSegElems;
-            const WT *pg = wg_lane + off, *pu = wu_lane + off;
-            uint4 *dst = wring + stage * (2 * kUnitChunks * 32);
+    // requests the gate and up chunks of unit (r, seg) into ring stage `stage`
+    auto request_unit = [&](int r, int seg, int stage) {
+        int chan;
+        if constexpr (FUSED) {
+            const int R = bx + nx * r;
+            const int grp = table[R >> lb];
+            if (lane == 0) ugrp_s[r][seg] = (short)grp;
+            chan = (grp << lb) + (R & (b - 1));
+        } else {
+            chan = chan_s[r];
+        }
+        const size_t off = (size_t)chan * d + (size_t)seg * kSegElems;
+        const WT *pg = wg_lane + off, *pu = wu_lane + off;
+        uint4 *dst = wring + stage * (2 * kUnitChunks * 32);
 #pragma unroll
-            for (int j = 0; j < kUnitChunks; ++j) {
-                if (FULL || (ci.seg * kUnitChunks + j) * 32 + lane < chunks) {
-                    cp_async16(dst + j * 32, pg + j * 32 * E);
-                    cp_async16(dst + (kUnitChunks + j) * 32, pu + j * 32 * E);
-                }
+        for (int j = 0; j < kUnitChunks; ++j) {
+            if (FULL || (seg * kUnitChunks + j) * 32 + lane < chunks) {
+                cp_async16(dst + j * 32, pg + j * 32 * E);
+                cp_async16(dst + (kUnitChunks + j) * 32, pu + j * 32 * E);
             }
         }
+    };
+    auto issue_unit = [&](int stage) {
+        if (ci.u < nunits) request_unit(ci.r, ci.seg, stage);
         cp_async_commit();  // one group per unit, empty past the end, so the wait count stays fixed
         advance(ci);
     };
-#pragma unroll
-    for (int i = 0; i < kUnitStages; ++i) issue_unit(i);
-    int stage = 0;
     // When the number of segments divides the number of warps, a warp meets the same segment in every
     // unit and its slice of h is loaded once; otherwise it is fetched (from L1) per unit.
     const bool fixed_seg = kGatherWarps % nseg == 0;
@@ -125,16 +203,13 @@ ffn_gather_kernel(const WT *__restrict__ Wg, const WT *__restrict__ Wu, const WT
             }
         }
     };
-    if (fixed_seg) load_h(cc.seg);
-#pragma unroll 1
-    for (; cc.u < nunits; advance(cc)) {
-        if (!fixed_seg) load_h(cc.seg);
-        cp_async_wait<kUnitStages - 1>();
+    // dot products of the unit in ring stage `stage` with the h slice in hv; lane 0 files them under (r, seg)
+    auto fold_unit = [&](int r, int seg, int stage) {
         const uint4 *src = wring + stage * (2 * kUnitChunks * 32);
         float g = 0.f, up = 0.f;
 #pragma unroll
         for (int j = 0; j < kUnitChunks; ++j) {
-            if (FULL || (cc.seg * kUnitChunks + j) * 32 + lane < chunks) {
+            if (FULL || (seg * kUnitChunks + j) * 32 + lane < chunks) {
                 float wg[E], wu[E];
                 Chunk<WT>::widen(src[j * 32], wg);
                 Chunk<WT>::widen(src[(kUnitChunks + j) * 32], wu);
@@ -142,12 +217,47 @@ ffn_gather_kernel(const WT *__restrict__ Wg, const WT *__restrict__ Wu, const WT
                 for (int e = 0; e < E; ++e) { g = fmaf(wg[e], hv[j][e], g); up = fmaf(wu[e], hv[j][e], up); }
             }
         }
+        return make_float2(g, up);
+    };
+    if (fixed_seg) load_h(cc.seg);
+    if constexpr (FUSED) bar_sync<2, kFusedThreads>();   // the table holds the first iteration's support
+#pragma unroll
+    for (int i = 0; i < kUnitStages; ++i) issue_unit(i);
+    int stage = 0;
+#pragma unroll 1
+    for (; cc.u < nunits; advance(cc)) {
+        if (!fixed_seg) load_h(cc.seg);
+        cp_async_wait<kUnitStages - 1>();
+        float2 gu = fold_unit(cc.r, cc.seg, stage);
         issue_unit(stage);  // refill the stage just consumed (its values were used above)
         stage = stage + 1 == kUnitStages ? 0 : stage + 1;
-        g = warp_sum(g); up = warp_sum(up);
-        if (lane == 0) { red[cc.r][cc.seg][0] = g; red[cc.r][cc.seg][1] = up; }
+        gu.x = warp_sum(gu.x); gu.y = warp_sum(gu.y);
+        if (lane == 0) { red[cc.r][cc.seg][0] = gu.x; red[cc.r][cc.seg][1] = gu.y; }
     }
     cp_async_wait<0>();
+
+    if constexpr (FUSED) {
+        bar_sync<3, kFusedThreads>();   // the recovery has finished: the table is final
+        if (tid < nrows) {
+            const int R = bx + nx * tid;
+            bad_s[tid] = 0;
+            chan_s[tid] = (table[R >> lb] << lb) + (R & (b - 1));
+        }
+        cta_sync();
+        // units that were requested for a group that has since left the slot: once more, one at a time
+        // (few: the rows requested early belong to the largest entries of the first iteration)
+#pragma unroll 1
+        for (Cursor c2{warp, warp / nseg, warp % nseg}; c2.u < nunits; advance(c2)) {
+            if ((int)ugrp_s[c2.r][c2.seg] == (chan_s[c2.r] >> lb)) continue;
+            if (!fixed_seg) load_h(c2.seg);
+            request_unit(c2.r, c2.seg, 0);
+            cp_async_commit();
+            cp_async_wait<0>();
+            float2 gu = fold_unit(c2.r, c2.seg, 0);
+            gu.x = warp_sum(gu.x); gu.y = warp_sum(gu.y);
+            if (lane == 0) { red[c2.r][c2.seg][0] = gu.x; red[c2.r][c2.seg][1] = gu.y; }
+        }
+    }
 
     // ---- down rows: thread i owns chunks i, i + 512, ... of every row; lane slots of the warp ring
     const WT *wd_thread = Wdt + tid * E;
@@ -167,13 +277,13 @@ ffn_gather_kernel(const WT *__restrict__ Wg, const WT *__restrict__ Wu, const WT
 #pragma unroll 1
     for (int r = 0; r < DR; ++r) issue_down();
 
-    __syncthreads();
+    cta_sync();
     if (tid < nrows) {
         float g = 0.f, up = 0.f;
         for (int sgm = 0; sgm < nseg; ++sgm) { g += red[tid][sgm][0]; up += red[tid][sgm][1]; }
-        a_s[tid] = silu(g) * up;
+        a_s[tid] = bad_s[tid] ? 0.f : silu(g) * up;
     }
-    __syncthreads();
+    cta_sync();
 
     float acc[CPT][E];
 #pragma unroll
@@ -285,22 +395,33 @@ cs_status launch_check_support(cs_plan *plan, const int32_t *support, int B, cud
 }
 
 // Picks the instantiation: chunks per thread in the down phase, and whether rows need bounds checks.
-template <typename WT>
+template <typename WT, bool FUSED>
 static void launch_gather_kernel(dim3 grid, cudaStream_t st, int cpt, int chunks, const WT *Wg, const WT *Wu,
-                                 const WT *Wd, const float *h, const int32_t *sup, int d, int b, int k,
-                                 float *partial) {
+                                 const WT *Wd, const float *h, const int32_t *sup, int d, int b, int k, int G,
+                                 float *partial, DeviceStatus *status, int check, const FusedArgs &fa) {
     const bool full = chunks % kGatherThreads == 0 && (cpt == 1 || cpt == 2 || cpt == 4);
-#define CS_GATHER_CASE(N, F)                                                                          \
-    launch_pdl(true, ffn_gather_kernel<WT, N, F>, grid, dim3(kGatherThreads), kRingBytes, st, Wg, Wu, Wd, h, sup, d, b, k, partial)
+    const int lb = b == 64 ? 6 : 7;
+#define CS_GATHER_CASE(N, F)                                                                              \
+    launch_pdl(true, ffn_gather_kernel<WT, N, F, FUSED>, grid, dim3(FUSED ? kFusedThreads : kGatherThreads), kRingBytes, st, \
+               Wg, Wu, Wd, h, sup, d, lb, k, G, partial, status, check, fa)
     if (cpt <= 1) { if (full) CS_GATHER_CASE(1, true); else CS_GATHER_CASE(1, false); }
     else if (cpt <= 2) { if (full) CS_GATHER_CASE(2, true); else CS_GATHER_CASE(2, false); }
     else { if (full) CS_GATHER_CASE(4, true); else CS_GATHER_CASE(4, false); }
 #undef CS_GATHER_CASE
 }
 
+// CTAs per token: one CTA per SM when a single token is in flight, never more than kGatherMaxRows rows per CTA.
+static int gather_nx(int sm_count, int nb, int rows_total, int nx_max) {
+    int nx = max(sm_count / nb, (rows_total + kGatherMaxRows - 1) / kGatherMaxRows);
+    return max(1, min(nx, min(rows_total, nx_max)));
+}
+
+// fa == NULL: supports given (`check`: validate them on the device).  Otherwise the fused step: fa holds the
+// recovery's inputs and outputs for all B tokens and `support` is unused.
 template <typename WT>
 static cs_status gather_typed(cs_plan *plan, const cs_layer *L, const float *h, const int32_t *support,
-                              int B, const float *residual, float *out, cudaStream_t st) {
+                              int B, const float *residual, float *out, int check, const FusedArgs *fa,
+                              cudaStream_t st) {
     const cs_config &c = plan->cfg;
     constexpr int E = Chunk<WT>::kElems;
     const int rows_total = c.k * c.group;
@@ -309,15 +430,23 @@ static cs_status gather_typed(cs_plan *plan, const cs_layer *L, const float *h, 
              *Wd = static_cast<const WT *>(L->Wd_t);
     for (int t0 = 0; t0 < B; t0 += kGatherMaxTokens) {
         const int nb = min(kGatherMaxTokens, B - t0);
-        // one CTA per SM when a single token is in flight, never more than kGatherMaxRows rows per CTA
-        int nx = max(plan->sm_count / nb, (rows_total + kGatherMaxRows - 1) / kGatherMaxRows);
-        nx = max(1, min(nx, min(rows_total, plan->nx_max)));
+        const int nx = gather_nx(plan->sm_count, nb, rows_total, plan->nx_max);
         dim3 grid(nx, nb);
         const float *hp = h + (size_t)t0 * c.d;
-        const int32_t *sp = support + (size_t)t0 * c.k;
         {
             StageTimer timer(plan, CS_STAGE_EXEC, st);
-            launch_gather_kernel<WT>(grid, st, cpt, c.d / E, Wg, Wu, Wd, hp, sp, c.d, c.group, c.k, plan->partial);
+            if (fa != nullptr) {
+                FusedArgs f = *fa;
+                f.y += (size_t)t0 * c.m;
+                if (f.support != nullptr) f.support += (size_t)t0 * c.k;
+                if (f.z != nullptr) f.z += (size_t)t0 * c.k;
+                if (f.resid != nullptr) f.resid += t0;
+                launch_gather_kernel<WT, true>(grid, st, cpt, c.d / E, Wg, Wu, Wd, hp, nullptr, c.d, c.group, c.k, plan->G,
+                                               plan->partial, plan->status, 0, f);
+            } else {
+                launch_gather_kernel<WT, false>(grid, st, cpt, c.d / E, Wg, Wu, Wd, hp, support + (size_t)t0 * c.k, c.d,
+                                                c.group, c.k, plan->G, plan->partial, plan->status, check, FusedArgs{});
+            }
         }
         plan->launches++;
         CS_CUDA_TRY(plan, cudaGetLastError());
@@ -334,23 +463,53 @@ static cs_status gather_typed(cs_plan *plan, const cs_layer *L, const float *h, 
 }
 
 // The ring needs more dynamic shared memory than the default limit: opt in once per kernel.
+template <typename WT, int N>
+static cudaError_t gather_attrs(bool fused_too) {
+    cudaError_t e = cudaFuncSetAttribute(ffn_gather_kernel<WT, N, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kRingBytes);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(ffn_gather_kernel<WT, N, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kRingBytes);
+    if (e == cudaSuccess && fused_too)
+        e = cudaFuncSetAttribute(ffn_gather_kernel<WT, N, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kRingBytes);
+    if (e == cudaSuccess && fused_too)
+        e = cudaFuncSetAttribute(ffn_gather_kernel<WT, N, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kRingBytes);
+    return e;
+}
+static cudaError_t gather_attrs_all(bool fused_too) {
+    cudaError_t e = gather_attrs<__nv_bfloat16, 1>(fused_too);
+    if (e == cudaSuccess) e = gather_attrs<__nv_bfloat16, 2>(fused_too);
+    if (e == cudaSuccess) e = gather_attrs<__nv_bfloat16, 4>(fused_too);
+    if (e == cudaSuccess) e = gather_attrs<float, 1>(fused_too);
+    if (e == cudaSuccess) e = gather_attrs<float, 2>(fused_too);
+    if (e == cudaSuccess) e = gather_attrs<float, 4>(fused_too);
+    return e;
+}
+
 cs_status prepare_ffn_gather(cs_plan *plan) {
-#define CS_GATHER_ATTR(WT, N)                                                                       \
-    CS_CUDA_TRY(plan, cudaFuncSetAttribute(ffn_gather_kernel<WT, N, true>,                          \
-                                           cudaFuncAttributeMaxDynamicSharedMemorySize, kRingBytes)); \
-    CS_CUDA_TRY(plan, cudaFuncSetAttribute(ffn_gather_kernel<WT, N, false>,                         \
-                                           cudaFuncAttributeMaxDynamicSharedMemorySize, kRingBytes))
-    CS_GATHER_ATTR(__nv_bfloat16, 1); CS_GATHER_ATTR(__nv_bfloat16, 2); CS_GATHER_ATTR(__nv_bfloat16, 4);
-    CS_GATHER_ATTR(float, 1); CS_GATHER_ATTR(float, 2); CS_GATHER_ATTR(float, 4);
-#undef CS_GATHER_ATTR
+    CS_CUDA_TRY(plan, gather_attrs_all(true));
     return CS_OK;
 }
 
 cs_status launch_ffn_gather(cs_plan *plan, const cs_layer *layer, const float *h, const int32_t *support,
-                            int B, const float *residual, float *out, cudaStream_t st) {
+                            int B, const float *residual, float *out, bool check, cudaStream_t st) {
     if (plan->cfg.w_dtype == CS_BF16)
-        return gather_typed<__nv_bfloat16>(plan, layer, h, support, B, residual, out, st);
-    return gather_typed<float>(plan, layer, h, support, B, residual, out, st);
+        return gather_typed<__nv_bfloat16>(plan, layer, h, support, B, residual, out, check, nullptr, st);
+    return gather_typed<float>(plan, layer, h, support, B, residual, out, check, nullptr, st);
+}
+
+bool fused_step_ok(const cs_plan *plan) { return plan->cfg.k <= kFusedMaxK && plan->G <= 32 * kFusedNW; }
+
+// Recovery of y (plan->gram must hold the layer's matrix: the sketch launch before formed it) and the
+// gather FFN on its result, in one launch per chunk of tokens.
+cs_status launch_recover_gather(cs_plan *plan, const cs_layer *layer, const float *h, const float *y, int B,
+                                const float *residual, float *out, int32_t *support, float *z, float *resid,
+                                cudaStream_t st) {
+    FusedArgs fa;
+    fa.Phi = layer->Phi; fa.gram = plan->gram; fa.y = y; fa.mu = layer->mu;
+    fa.m = plan->cfg.m; fa.T = plan->cfg.T; fa.pitch = gram_pitch(plan->G);
+    fa.support = support; fa.z = z; fa.resid = resid;
+    if (plan->cfg.w_dtype == CS_BF16)
+        return gather_typed<__nv_bfloat16>(plan, layer, h, nullptr, B, residual, out, 0, &fa, st);
+    return gather_typed<float>(plan, layer, h, nullptr, B, residual, out, 0, &fa, st);
 }
 
 
@@ -378,14 +537,7 @@ static cudaError_t static_setup(int dev) {
     int sms = 0;
     e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     if (e != cudaSuccess) return e;
-#define CS_STATIC_ATTR(WT, N)                                                                        \
-    if (e == cudaSuccess)                                                                            \
-        e = cudaFuncSetAttribute(ffn_gather_kernel<WT, N, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kRingBytes); \
-    if (e == cudaSuccess)                                                                            \
-        e = cudaFuncSetAttribute(ffn_gather_kernel<WT, N, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kRingBytes)
-    CS_STATIC_ATTR(__nv_bfloat16, 1); CS_STATIC_ATTR(__nv_bfloat16, 2); CS_STATIC_ATTR(__nv_bfloat16, 4);
-    CS_STATIC_ATTR(float, 1); CS_STATIC_ATTR(float, 2); CS_STATIC_ATTR(float, 4);
-#undef CS_STATIC_ATTR
+    if (e == cudaSuccess) e = gather_attrs_all(false);
     if (e != cudaSuccess) return e;
     g_static_sms[dev] = sms;
     g_static_ptr[dev] = static_cast<float *>(p);
@@ -401,7 +553,8 @@ static cudaError_t static_launch(const cs_config &c, const cs_layer *L, const fl
     const WT *Wg = static_cast<const WT *>(L->W_gate), *Wu = static_cast<const WT *>(L->W_up),
              *Wd = static_cast<const WT *>(L->Wd_t);
     dim3 grid(nx, B);
-    launch_gather_kernel<WT>(grid, st, cpt, c.d / E, Wg, Wu, Wd, h, support, c.d, c.group, c.k, partial);
+    launch_gather_kernel<WT, false>(grid, st, cpt, c.d / E, Wg, Wu, Wd, h, support, c.d, c.group, c.k, c.d_ff / c.group,
+                                    partial, static_cast<DeviceStatus *>(nullptr), 0, FusedArgs{});
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     dim3 rgrid((c.d / 4 + kReduceCols - 1) / kReduceCols, B);
@@ -422,6 +575,11 @@ extern "C" cs_status cs_ffn_exec_static(const cs_config *cfg, const cs_layer *la
         return CS_ERR_SHAPE;
     if ((cfg->group != 64 && cfg->group != 128) || cfg->d > kMaxD || cfg->d % 64 != 0 ||
         cfg->d_ff / cfg->group > kMaxG || (cfg->w_dtype != CS_F32 && cfg->w_dtype != CS_BF16))
+        return CS_ERR_UNSUPPORTED;
+    // the kernels move 16-byte chunks: the same alignment rule as cs_ffn_exec, checked before anything runs
+    auto misaligned = [](const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; };
+    if (misaligned(layer->W_gate) || misaligned(layer->W_up) || misaligned(layer->Wd_t) || misaligned(h) ||
+        misaligned(out) || (residual != nullptr && misaligned(residual)))
         return CS_ERR_UNSUPPORTED;
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kStaticMaxDevices) return CS_ERR_CUDA;

@@ -6,7 +6,11 @@ Tolerances (relative l2 unless noted):
              a token below that margin is "excused" and its output is compared against the oracle
              re-run with the library's support
   z          <= 1e-4
-  outputs    <= 1e-5 with float32 weights, <= 1e-2 with bfloat16 weights
+  outputs    <= 1e-5 with float32 weights, <= 1e-2 with bfloat16 weights (the stated bars), and beside
+             them the level the arithmetic actually reaches, so that a dropped k block or a wrong
+             remainder operand cannot hide under the loose bar: <= 1e-4 wherever the activations are
+             float32 (the oracle reads the same stored bfloat16 weights, so weight rounding is no
+             error source), <= 5e-3 for the prompt-level path, whose activations are bfloat16
 """
 from __future__ import annotations
 
@@ -22,6 +26,8 @@ from gen import workloads as W
 GAP_TOL = 1e-4
 Z_TOL = 1e-4
 OUT_TOL = {"f32": 1e-5, "bf16": 1e-2}
+TIGHT_TOL = {"f32": 1e-5, "bf16": 1e-4}   # float32 activations
+PROMPT_TIGHT_TOL = 5e-3                   # bfloat16 activations in and out, bfloat16 between the two GEMMs
 
 
 def rel(a, b) -> float:
@@ -91,7 +97,7 @@ def compare_layer_step(cfg: W.Config, L_dev: W.Layer, plan: cs.Plan, x_cpu: torc
                             add_residual=add_residual)
     sup = sup.cpu().numpy(); z = z.cpu().numpy(); out = x_out.cpu().numpy(); resid = resid.cpu().numpy()
     B = x_cpu.shape[0]
-    tol = OUT_TOL[cfg.w_dtype]
+    tol = min(OUT_TOL[cfg.w_dtype], TIGHT_TOL[cfg.w_dtype])
     excused = 0
     forced_rows = []
     rep = StepReport(B, 0, 0.0, 0.0, 0.0)

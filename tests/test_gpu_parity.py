@@ -7,8 +7,8 @@ import torch
 import oracle
 import paper_2604_14156_b200 as cs
 from gen import rng, workloads as W
-from parity_util import (GAP_TOL, OUT_TOL, Z_TOL, compare_layer_step, device_layer, make_plan, recovery_matches,
-                         rel)
+from parity_util import (GAP_TOL, OUT_TOL, PROMPT_TIGHT_TOL, TIGHT_TOL, Z_TOL, compare_layer_step, device_layer,
+                         make_plan, recovery_matches, rel)
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda"
@@ -222,8 +222,8 @@ def test_ffn_exec_matches_oracle_on_given_supports(name, B):
     assert plan.device_status() == 0
     for t in range(B):
         ref = oracle.ffn(Lc.W_gate, Lc.W_up, Lc.Wd_t, cfg.group, tk.h[t], tk.planted[t])
-        assert rel(out0[t], ref) <= OUT_TOL[cfg.w_dtype]
-        assert rel(out[t], ref + res[t].double().numpy()) <= OUT_TOL[cfg.w_dtype]
+        assert rel(out0[t], ref) <= TIGHT_TOL[cfg.w_dtype]
+        assert rel(out[t], ref + res[t].double().numpy()) <= TIGHT_TOL[cfg.w_dtype]
 
 
 def test_ffn_exec_all_groups_is_the_dense_ffn():
@@ -255,6 +255,76 @@ def test_ffn_exec_flags_invalid_supports():
     cs.cs_ffn_exec(plan, lay, h, bad)
     assert plan.device_status() == 4
     assert plan.device_status() == 0  # reading clears it
+
+
+def test_ffn_exec_out_of_range_groups_are_skipped_not_read():
+    """A group index outside [0, G) never becomes an address: it is flagged, its channels contribute
+    zero, and every other entry and token is computed as usual (gather path and tensor-core path)."""
+    for name, B in (("tiny_f32", 3), ("l2_7b_b64", 3), ("l2_7b_b64", 7)):
+        cfg = W.CONFIGS[name]
+        L = _layer(cfg)
+        Lc = L.to("cpu")
+        tk = W.make_tokens(cfg, L.A, B=B)
+        plan = make_plan(cfg, max_tokens=B)
+        sup = tk.planted.clone()
+        sup[1, 0] = -3
+        sup[1, cfg.k - 1] = cfg.G + 5
+        out = cs.cs_ffn_exec(plan, device_layer(plan, L), tk.h.to(DEV), sup.to(DEV)).cpu().numpy()
+        assert plan.device_status() == 4
+        for t in range(B):
+            valid = sup[t][(sup[t] >= 0) & (sup[t] < cfg.G)]
+            ref = oracle.ffn(Lc.W_gate, Lc.W_up, Lc.Wd_t, cfg.group, tk.h[t], valid)
+            assert rel(out[t], ref) <= TIGHT_TOL[cfg.w_dtype], (name, B, t)
+        plan.close()
+
+
+def test_recover_non_finite_row_stays_in_its_row():
+    """A NaN in one token's sketch: that token's outputs are k valid, ascending, distinct indices (its
+    values are NaN) and the status word reports it; the neighbouring tokens are untouched."""
+    for name in ("tiny_f32", "l2_7b_b64"):
+        cfg = W.CONFIGS[name]
+        Phi = rng.normal(cfg.seed, (W.T_PHI, 0), (cfg.m, cfg.G), dtype=torch.float32, scale=cfg.m ** -0.5)
+        mu = W.spectral_step(Phi)
+        y = rng.normal(cfg.seed, (81,), (3, cfg.m), dtype=torch.float32)
+        y[1, cfg.m // 2] = float("nan")
+        plan = make_plan(cfg, max_tokens=3)
+        guard = torch.full((5, cfg.k), -7, dtype=torch.int32, device=DEV)   # rows 1..3 are the outputs
+        zg = torch.full((5, cfg.k), 123.0, dtype=torch.float32, device=DEV)
+        resid = torch.empty(3, dtype=torch.float32, device=DEV)
+        Phi_d, y_d = Phi.to(DEV), y.to(DEV)   # named: a temporary would be freed (and reused) before the launch
+        st = plan.lib.cs_recover(plan.handle, Phi_d.data_ptr(), float(mu), y_d.data_ptr(), 3,
+                                 guard[1:4].data_ptr(), zg[1:4].data_ptr(), resid.data_ptr(),
+                                 torch.cuda.current_stream().cuda_stream)
+        assert st == 0
+        assert plan.device_status() == 5
+        g = guard.cpu().numpy(); zz = zg.cpu().numpy()
+        assert (g[0] == -7).all() and (g[4] == -7).all() and (zz[0] == 123.0).all() and (zz[4] == 123.0).all()
+        for row, t in ((1, 0), (3, 2)):
+            ref = oracle.iht(Phi, y[t], cfg.k, cfg.T, mu)
+            assert recovery_matches(g[row], zz[row], resid[t].item(), ref, Phi.numpy(), y[t].numpy(), (name, t))
+        assert (np.diff(g[2]) > 0).all() and g[2][0] >= 0 and g[2][-1] < cfg.G
+        plan.close()
+
+
+def test_layer_step_non_finite_token_does_not_disturb_the_others():
+    """The whole step with a NaN hidden state in the middle token (gather path, fused recovery)."""
+    cfg = W.CONFIGS["tiny_f32"].with_(B=3)
+    L = _layer(cfg)
+    tk = W.make_tokens(cfg, L.A, B=3)
+    x = tk.h.clone()
+    x[1, 7] = float("nan")
+    plan = make_plan(cfg, max_tokens=3)
+    out, sup, z, resid = cs.cs_layer_step(plan, device_layer(plan, L), x.to(DEV))
+    torch.cuda.synchronize()
+    assert plan.device_status() == 5
+    ref = oracle.layer_step(L.to("cpu"), tk.h, group=cfg.group, k=cfg.k, T=cfg.T)
+    sup = sup.cpu().numpy(); out = out.cpu().numpy()
+    for t in (0, 2):
+        if ref.min_gap[t] > GAP_TOL:
+            assert np.array_equal(sup[t], ref.support[t])
+            assert rel(out[t], ref.x_out[t]) <= TIGHT_TOL["f32"]
+    assert (np.diff(sup[1]) > 0).all() and sup[1][0] >= 0 and sup[1][-1] < cfg.G
+    plan.close()
 
 
 def test_call_errors_come_back_as_codes():
@@ -440,9 +510,10 @@ def test_ffn_exec_tensor_path_matches_oracle(B):
     res = rng.normal(cfg.seed, (79,), (B, cfg.d), dtype=torch.float32)
     out = cs.cs_ffn_exec(plan, lay, tk.h.to(DEV), tk.planted.to(DEV), residual=res.to(DEV)).cpu().numpy()
     assert plan.device_status() == 0
-    for t in (range(B) if B <= 16 else sorted({0, 1, B // 2, B - 2, B - 1})):
+    for t in range(B):   # every token
         ref = oracle.ffn(Lc.W_gate, Lc.W_up, Lc.Wd_t, cfg.group, tk.h[t], tk.planted[t])
-        assert rel(out[t] - res[t].numpy(), ref) <= OUT_TOL["bf16"], t
+        err = rel(out[t].astype(np.float64) - res[t].double().numpy(), ref)
+        assert err <= OUT_TOL["bf16"] and err <= TIGHT_TOL["bf16"], (t, err)
 
 
 @pytest.mark.parametrize("B", [4, 5, 9])
@@ -464,14 +535,15 @@ def test_ffn_exec_tensor_path_skips_unused_groups():
     sup = torch.tensor([[1, 40, 85], [1, 2, 85], [0, 40, 41]], dtype=torch.int32).repeat(7, 1)[:20].contiguous()
     plan = make_plan(cfg, max_tokens=20)
     out = cs.cs_ffn_exec(plan, device_layer(plan, L), tk.h.to(DEV), sup.to(DEV)).cpu().numpy()
-    for t in (0, 1, 2, 19):
+    for t in range(20):
         ref = oracle.ffn(Lc.W_gate, Lc.W_up, Lc.Wd_t, cfg.group, tk.h[t], sup[t])
-        assert rel(out[t], ref) <= OUT_TOL["bf16"], t
+        assert rel(out[t], ref) <= TIGHT_TOL["bf16"], t
 
 
 @pytest.mark.parametrize("k", W.PROMPT_K_SWEEP)
 def test_ffn_exec_shared_parity(k):
-    """Prompt-level variant at full size: 2048 tokens, one shared support; sampled tokens against the oracle."""
+    """Prompt-level variant at full size: 2048 tokens, one shared support; the first, a middle and the
+    last token of each of the sixteen 128-token tiles against the oracle."""
     cfg = W.CONFIGS["l2_13b_prompt"].with_(k=k)
     L = _layer(cfg)
     Lc = L.to("cpu")
@@ -485,9 +557,14 @@ def test_ffn_exec_shared_parity(k):
     assert plan.device_status() == 0
     out = out.float().cpu().numpy()
     s = sup.cpu().numpy()
-    for t in (0, 1, 127, 128, 1000, 2046, 2047):
-        ref = oracle.ffn(Lc.W_gate, Lc.W_up, Lc.Wd_t, cfg.group, tk.h[t].double().numpy(), s)
-        assert rel(out[t], ref) <= OUT_TOL["bf16"], t
+    worst = 0.0
+    for tile in range(cfg.B // 128):
+        for t in (128 * tile, 128 * tile + 37 + tile, 128 * tile + 127):
+            ref = oracle.ffn(Lc.W_gate, Lc.W_up, Lc.Wd_t, cfg.group, tk.h[t].double().numpy(), s)
+            err = rel(out[t], ref)
+            assert err <= OUT_TOL["bf16"] and err <= PROMPT_TIGHT_TOL, (t, err)
+            worst = max(worst, err)
+    print(f"k={k}: worst relative error over 48 tokens {worst:.2e}")
 
 
 def test_ffn_exec_shared_ragged_prompt_length():
@@ -501,7 +578,7 @@ def test_ffn_exec_shared_ragged_prompt_length():
     assert plan.device_status() == 0
     for t in (0, 127, 128, 255, 256, 332):
         ref = oracle.ffn(Lc.W_gate, Lc.W_up, Lc.Wd_t, cfg.group, tk.h[t].double().numpy(), sup.cpu().numpy())
-        assert rel(out[t], ref) <= OUT_TOL["bf16"], t
+        assert rel(out[t], ref) <= PROMPT_TIGHT_TOL, t
 
 
 def test_ffn_exec_shared_random_shapes():
@@ -522,7 +599,7 @@ def test_ffn_exec_shared_random_shapes():
         assert plan.device_status() == 0
         for t in sorted({0, n // 2, n - 1, min(n - 1, 127), min(n - 1, 128)}):
             ref = oracle.ffn(Lc.W_gate, Lc.W_up, Lc.Wd_t, cfg.group, tk.h[t].double().numpy(), sup.cpu().numpy())
-            assert rel(out[t], ref) <= OUT_TOL["bf16"], (trial, G, k, d, n, t)
+            assert rel(out[t], ref) <= PROMPT_TIGHT_TOL, (trial, G, k, d, n, t)
         plan.close()
 
 
@@ -664,6 +741,27 @@ def test_layer_step_host_matches_device_entry(name, B, pinned):
             torch.cuda.synchronize()
             want, _, _, _ = cs.cs_layer_step(plan, lay, tk.h.to(DEV))
             assert torch.equal(hout, want.cpu()), batch
+    plan.close()
+
+
+def test_layer_step_host_chained_through_one_buffer():
+    """Three layers chained through ONE pinned buffer with no synchronisation in between: layer i stores
+    its result into the buffer layer i + 1 reads, so the staging load must respect stream order."""
+    cfg = W.CONFIGS["l3_8b_stack"].with_(B=2)
+    plan = make_plan(cfg, max_tokens=2)
+    Ls = [_layer(cfg, i) for i in range(3)]
+    lays = [device_layer(plan, L) for L in Ls]
+    x0 = W.make_tokens(cfg, Ls[0].A, B=2).h
+    buf = torch.empty((2, cfg.d), dtype=torch.float32).pin_memory()
+    for rep in range(3):
+        buf.copy_(x0)
+        for lay in lays:
+            cs.cs_layer_step_host(plan, lay, buf, buf)
+        torch.cuda.synchronize()
+        x = x0.to(DEV)
+        for lay in lays:
+            x, _, _, _ = cs.cs_layer_step(plan, lay, x)
+        assert torch.equal(buf, x.cpu()), rep
     plan.close()
 
 
