@@ -262,6 +262,20 @@ cs_status cs_plan_set_crossover(cs_plan *plan, int32_t tokens);
 int32_t cs_plan_crossover(const cs_plan *plan);
 
 /*
+ * Speculative start of the actuator at small batches (Sec. 5: the support is estimated while the
+ * model runs; Sec. 15 asks that the sensing stage be accounted for, not hidden).  Off by default.  When
+ * on, cs_layer_step below the regime crossover runs sketch and recovery in ONE launch and starts the
+ * gather FFN's weight stream on the support of the FIRST iterate while the remaining iterations
+ * run; rows requested for a group that later leaves the support are fetched again, so the supports
+ * are those of the plain path and the outputs agree with it to rounding (the rows of a token are
+ * dealt to one CTA fewer, which changes the order of the partial sums).  It needs k <= 32, G <= 128 and m <= 32
+ * (CS_ERR_UNSUPPORTED otherwise).  On the shapes measured so far it is not faster than the plain chain
+ * of launches (the recovery it overlaps costs less than the bookkeeping it adds), which is why it
+ * is opt-in.
+ */
+cs_status cs_plan_set_speculative(cs_plan *plan, int32_t on);
+
+/*
  * Stage timing (the paper asks for sensing / recovery overhead to be reported apart from the
  * sparse kernel itself, Sec. 15 metric suite).  While enabled, every launch of a stage is bracketed
  * by CUDA events on the call's stream.  cs_plan_stage_times synchronises `stream` and returns the

@@ -73,6 +73,8 @@ def load_library():
     lib.cs_plan_enable_timing.argtypes = [vp, i32]
     lib.cs_plan_set_crossover.argtypes = [vp, i32]
     lib.cs_plan_set_crossover.restype = ctypes.c_int
+    lib.cs_plan_set_speculative.argtypes = [vp, i32]
+    lib.cs_plan_set_speculative.restype = ctypes.c_int
     lib.cs_plan_crossover.argtypes = [vp]
     lib.cs_plan_crossover.restype = ctypes.c_int32
     lib.cs_plan_stage_times.argtypes = [vp, vp, ctypes.POINTER(f32 * 5)]
@@ -153,6 +155,10 @@ class Plan:
 
     def set_crossover(self, tokens: int):
         self.check(self.lib.cs_plan_set_crossover(self.handle, int(tokens)), "cs_plan_set_crossover")
+
+    def set_speculative(self, on: bool = True):
+        """Small batches: start the gather FFN on the recovery's first iterate (see include/cs.h)."""
+        self.check(self.lib.cs_plan_set_speculative(self.handle, int(on)), "cs_plan_set_speculative")
 
     def enable_timing(self, on: bool = True):
         self.check(self.lib.cs_plan_enable_timing(self.handle, int(on)), "cs_plan_enable_timing")

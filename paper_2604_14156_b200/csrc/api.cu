@@ -84,6 +84,8 @@ cs_status cs_plan_create(const cs_config *cfg, cs_plan **out) {
     alloc((void **)&p->sup_buf, nt * cfg->k * sizeof(int32_t));
     alloc((void **)&p->partial, (size_t)kGatherMaxTokens * p->nx_max * cfg->d * sizeof(float));
     alloc((void **)&p->gram, (size_t)kMaxG * kMaxG * sizeof(float));
+    alloc((void **)&p->slot_table, nt * kSlotTablePitch * sizeof(int32_t));
+    alloc((void **)&p->ticket, nt * sizeof(unsigned));
     alloc((void **)&p->hbar, (size_t)cfg->d * sizeof(float));
     alloc((void **)&p->colsum, (size_t)p->mean_row_blocks * cfg->d * sizeof(float));
     alloc((void **)&p->status, sizeof(DeviceStatus));
@@ -116,6 +118,9 @@ cs_status cs_plan_create(const cs_config *cfg, cs_plan **out) {
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p->ev_fork, cudaEventDisableTiming);
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p->ev_join, cudaEventDisableTiming);
     if (e == cudaSuccess) e = cudaMemset(p->status, 0, sizeof(DeviceStatus));
+    if (e == cudaSuccess) e = cudaMemset(p->ticket, 0, nt * sizeof(unsigned));
+    if (e == cudaSuccess) e = cudaMemset(p->slot_table, 0, nt * kSlotTablePitch * sizeof(int32_t));
+    if (e == cudaSuccess && prepare_sketch(p) != CS_OK) e = cudaErrorUnknown;
     if (e == cudaSuccess && prepare_ffn_gather(p) != CS_OK) e = cudaErrorUnknown;
     if (e == cudaSuccess && p->mma_ok && prepare_ffn_mma(p) != CS_OK) e = cudaErrorUnknown;
     if (e != cudaSuccess) {
@@ -129,7 +134,7 @@ cs_status cs_plan_create(const cs_config *cfg, cs_plan **out) {
 cs_status cs_plan_destroy(cs_plan *p) {
     if (p == nullptr) return CS_ERR_NULL;
     cudaFree(p->n_buf); cudaFree(p->y_buf); cudaFree(p->sup_buf);
-    cudaFree(p->partial); cudaFree(p->gram); cudaFree(p->hbar); cudaFree(p->colsum);
+    cudaFree(p->partial); cudaFree(p->gram); cudaFree(p->slot_table); cudaFree(p->ticket); cudaFree(p->hbar); cudaFree(p->colsum);
     cudaFree(p->status); cudaFree(p->x_host_in); cudaFree(p->x_host_out);
     cudaFree(p->mask); cudaFree(p->gmask); cudaFree(p->counts); cudaFree(p->offsets); cudaFree(p->token_ids); cudaFree(p->glist);
     cudaFree(p->nu); cudaFree(p->x_bf16); cudaFree(p->act); cudaFree(p->mma_partial);
@@ -300,12 +305,17 @@ cs_status cs_layer_step(cs_plan *plan, const cs_layer *layer, const float *x, in
             return r;
         }, layer->rms_gamma);
     }
+    const bool gather = !plan->mma_ok || B < plan->mma_min_tokens;
+    if (gather && plan->speculative && sketch_recover_ok(plan) && !plan->timing) {
+        // Opt-in (cs_plan_set_speculative): sketch and recovery in one launch, and the gather FFN behind it
+        // starts its weight stream on the first iterate while the other iterations run.  (Not while stages
+        // are being timed: event records between the launches would serialise them.)
+        s = launch_sketch_recover(plan, layer, x, B, plan->y_buf, norm ? plan->n_buf : nullptr, support_out, z_out, resid_out, st);
+        if (s != CS_OK) return s;
+        return launch_ffn_gather_spec(plan, layer, n, B, layer->add_residual ? x : nullptr, x_out, st);
+    }
     s = launch_sketch(plan, layer->S, x, layer->rms_gamma, B, plan->y_buf, norm ? plan->n_buf : nullptr, layer->Phi, layer->mu, st);
     if (s != CS_OK) return s;
-    const bool gather = !plan->mma_ok || B < plan->mma_min_tokens;
-    if (gather && fused_step_ok(plan))   // recovery and gather FFN in one launch: the weight stream starts on the first iterate
-        return launch_recover_gather(plan, layer, n, plan->y_buf, B, layer->add_residual ? x : nullptr, x_out, support_out,
-                                     z_out, resid_out, st);
     s = launch_recover(plan, layer->Phi, layer->mu, plan->y_buf, B, sup, z_out, resid_out, true, st);
     if (s != CS_OK) return s;
     // supports produced by the recovery are valid by construction: no device check here
@@ -364,6 +374,13 @@ cs_status cs_plan_set_crossover(cs_plan *plan, int32_t tokens) {
 }
 
 int32_t cs_plan_crossover(const cs_plan *plan) { return plan != nullptr ? plan->mma_min_tokens : 0; }
+
+cs_status cs_plan_set_speculative(cs_plan *plan, int32_t on) {
+    if (plan == nullptr) return CS_ERR_NULL;
+    if (on && !sketch_recover_ok(plan)) return CS_ERR_UNSUPPORTED;
+    plan->speculative = on != 0;
+    return CS_OK;
+}
 
 cs_status cs_plan_enable_timing(cs_plan *plan, int32_t on) {
     if (plan == nullptr) return CS_ERR_NULL;

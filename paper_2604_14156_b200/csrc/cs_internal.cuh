@@ -15,6 +15,8 @@ constexpr int kMaxD = 8192;       // hidden size
 constexpr int kGatherThreads = 512;
 constexpr int kGatherMaxRows = 32;   // channel rows one gather CTA owns at most
 constexpr int kGatherMaxTokens = 16; // tokens per gather launch (scratch for partial sums)
+constexpr int kSlotTableSlots = 32;  // slots per token of the recovery's slot table (small-batch step) ...
+constexpr int kSlotTablePitch = 40;  // ... and ints per token: the slots, then a word that says "final"
 constexpr int kReduceGroups = 32;    // partial-sum groups of the deterministic cross-CTA reduction
 constexpr int kMmaMinTokens = 16;    // decode batches at least this large always run on the tensor cores; a plan
                                      // lowers the bound by its G / k (cs_plan_set_crossover overrides it)
@@ -37,6 +39,8 @@ struct cs_plan {
     int32_t *sup_buf;  // [max_tokens, k]
     float *partial;    // [kGatherMaxTokens, nx_max, d] partial down-projections of the gather path
     float *gram;       // [G, pitch] I - mu Phi^T Phi of the layer being recovered, pitch = 32 ceil(G/32)
+    int32_t *slot_table;  // [max_tokens, kSlotTablePitch] small-batch step: slot -> group of the recovery in flight
+    unsigned *ticket;     // [max_tokens] arrival counters of the sketch CTAs (zero between launches)
     float *hbar;       // [d] mean prompt hidden state
     float *colsum;     // [mean_row_blocks, d]
     cs::DeviceStatus *status;  // device status word
@@ -51,6 +55,7 @@ struct cs_plan {
     void *x_bf16;        // [2][max_tokens, d] bf16 activations: rounded value, then remainder
     void *act;           // [2][max_tokens, d_ff] bf16 SwiGLU activations over the group list (value, remainder)
     float *mma_partial;  // [slices, padded tokens, d] f32 partial down projections
+    int speculative;     // small batches: start the weight stream on the recovery's first iterate (opt-in)
     int mma_ok;          // shape qualifies for the tensor-core path
     int mma_min_tokens;  // smallest decode batch that takes it
     int mma_slices;      // most list slices the down GEMM is split into
@@ -109,11 +114,15 @@ cs_status launch_recover(cs_plan *plan, const float *Phi, float mu, const float 
 // check: validate the supports on the device (ascending, distinct, in range) inside the same launch
 cs_status launch_ffn_gather(cs_plan *plan, const cs_layer *layer, const float *h, const int32_t *support,
                             int B, const float *residual, float *out, bool check, cudaStream_t st);
-// the small-batch step in one launch: recovery of y beside the gather FFN that starts on its first iterate
-bool fused_step_ok(const cs_plan *plan);
-cs_status launch_recover_gather(cs_plan *plan, const cs_layer *layer, const float *h, const float *y, int B,
-                                const float *residual, float *out, int32_t *support, float *z, float *resid,
-                                cudaStream_t st);
+// The small-batch step: sketch and recovery in one launch, whose programmatic trigger fires when the
+// first iterate's slot table is in memory; the gather FFN launched behind it starts on that table,
+// follows the table while the iteration runs, and settles on the final one.
+bool sketch_recover_ok(const cs_plan *plan);
+cs_status prepare_sketch(cs_plan *plan);
+cs_status launch_sketch_recover(cs_plan *plan, const cs_layer *L, const float *x, int B, float *y, float *n_out,
+                                int32_t *support, float *z, float *resid, cudaStream_t st);
+cs_status launch_ffn_gather_spec(cs_plan *plan, const cs_layer *layer, const float *h, int B, const float *residual,
+                                 float *out, cudaStream_t st);
 cs_status prepare_ffn_gather(cs_plan *plan);
 cs_status launch_support_drift(cs_plan *plan, const int32_t *prev, const int32_t *cur, int B, int32_t *drift,
                                cudaStream_t st);

@@ -22,19 +22,17 @@
 // The partial d-vectors are summed in a fixed order by reduce_partials_kernel (deterministic,
 // no atomics), which also adds the residual.
 //
-// FUSED (cs_layer_step at small batches): the supports are not an input.  Four extra warps of every
-// CTA run the recovery of the CTA's token (recover_core.cuh; every CTA of a token repeats it, which
-// costs nothing that matters: a few KB from L2), and the 16 streaming warps start on the support of
-// the FIRST iteration while the other iterations run.  The recovery keeps its support as a table of
-// k stable slots (slot -> group) in shared memory; the streaming warps read the table when they
-// request a row and remember which group they requested.  The first iteration hands the slots out
-// by decreasing magnitude and rows are dealt to CTAs and requested in slot order, so the rows
-// requested first belong to the entries least likely to leave the support, and a slot that does
-// change costs every CTA at most one row (not one CTA all of its rows).  When the recovery has
-// finished, units whose remembered group is not the slot's final one are fetched and computed
-// again; the down phase only ever uses the final table.
-#include <type_traits>
-
+// SPEC (cs_layer_step at small batches): the supports are not an input; the recovery is still running
+// (in the launch before this one, whose programmatic trigger fired when the slot table of its FIRST
+// iterate was in global memory) while this kernel streams.  The recovery keeps its support as a
+// table of k stable slots (slot -> group); a 17th warp of every CTA keeps copying the table of the
+// CTA's token from global to shared memory, the streaming warps read that copy when they request a
+// row and remember which group they requested.  The first iteration hands the slots out by
+// decreasing magnitude and rows are dealt to CTAs and requested in slot order, so the rows requested
+// first belong to the entries least likely to leave the support, and a slot that does change costs
+// every CTA at most one row (not one CTA all of its rows).  After the gate/up pass the kernel waits
+// for the launch before it to complete, reads the final table, fetches and computes again the units
+// whose remembered group is not the slot's final one, and runs the down phase on the final table.
 #include "recover_core.cuh"
 
 namespace cs {
@@ -50,18 +48,19 @@ constexpr int kUnitStages = kWarpRing / kUnitBytes;        // 3 units in flight 
 constexpr int kLaneSlots = kWarpRing / (32 * 16);          // 24 chunks per lane in the down phase
 constexpr int kMaxSegs = kMaxD * 4 / (kUnitChunks * 32 * 16);  // 16 (f32 rows of 8192)
 
-// Recovery side of the fused kernel: G <= 128 entries on four warps, list form with up to 32 slots.
-constexpr int kFusedNW = 4, kFusedKC = 4;
-constexpr int kFusedMaxK = 8 * kFusedKC;
-constexpr int kFusedThreads = kGatherThreads + 32 * kFusedNW;
-struct FusedArgs {
-    const float *Phi, *gram, *y;   // [m,G], [G,pitch], [B,m]
-    float mu;
-    int m, T, pitch;
-    int32_t *support;              // [B,k] ascending (may be NULL)
-    float *z, *resid;              // [B,k], [B] (may be NULL)
-};
-struct NoSmem {};
+constexpr int kSpecThreads = kGatherThreads + 32;   // the streaming warps + the warp that follows the slot table
+constexpr uint32_t kFollowLimit = 1u << 16;         // polls of the table after which the following warp gives up
+
+__device__ __forceinline__ int ld_visible(const int32_t *p) {
+    int v;
+    asm volatile("ld.volatile.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ int ld_acquire(const int32_t *p) {
+    int v;
+    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
 
 __device__ __forceinline__ void cp_async16(void *smem_dst, const void *gmem_src) {
     const uint32_t s = static_cast<uint32_t>(__cvta_generic_to_shared(smem_dst));
@@ -75,11 +74,12 @@ template <int N> __device__ __forceinline__ void cp_async_wait() {
 // CPT = 16-byte chunks per thread and row in the down phase (row bytes / (512 * 16), rounded up).
 // FULL = every row is a whole number of units and of 512-chunk slices: no bounds checks inside.
 // check: the CTAs with blockIdx.x == 0 also validate their token's support row (ascending, distinct).
-template <typename WT, int CPT, bool FULL, bool FUSED>
-__global__ void __launch_bounds__(FUSED ? kFusedThreads : kGatherThreads, 1)
+// SPEC: `support` is the recovery's slot table, [tokens, kSlotTablePitch], still changing.
+template <typename WT, int CPT, bool FULL, bool SPEC>
+__global__ void __launch_bounds__(SPEC ? kSpecThreads : kGatherThreads, 1)
 ffn_gather_kernel(const WT *__restrict__ Wg, const WT *__restrict__ Wu, const WT *__restrict__ Wdt,
                   const float *__restrict__ h, const int32_t *__restrict__ support, int d, int lb, int k, int G,
-                  float *__restrict__ partial, DeviceStatus *status, int check, FusedArgs fa) {
+                  float *__restrict__ partial, DeviceStatus *status, int check) {
     constexpr int E = Chunk<WT>::kElems;
     constexpr int DR = kLaneSlots / CPT;               // down rows in flight per thread
     constexpr int kSegElems = kUnitChunks * 32 * E;    // elements of one row segment
@@ -88,8 +88,11 @@ ffn_gather_kernel(const WT *__restrict__ Wg, const WT *__restrict__ Wu, const WT
     __shared__ float a_s[kGatherMaxRows];
     __shared__ int chan_s[kGatherMaxRows];
     __shared__ int bad_s[kGatherMaxRows];   // row belongs to a group index outside [0, G): contributes nothing
-    __shared__ short ugrp_s[FUSED ? kGatherMaxRows : 1][FUSED ? kMaxSegs : 1];   // group each unit was requested for
-    __shared__ typename std::conditional<FUSED, RecoverSmem<kFusedNW, kFusedKC>, NoSmem>::type rs;
+    __shared__ short ugrp_s[SPEC ? kGatherMaxRows : 1][SPEC ? kMaxSegs : 1];   // group each unit was requested for
+    __shared__ int table_s[SPEC ? kSlotTableSlots : 1];                       // the slot table as last seen
+    __shared__ int done_s, final_s;                                           // pass over; table_s is the final table
+    __shared__ short stale_s[SPEC ? kGatherMaxRows * kMaxSegs : 1];           // units to fetch and fold once more
+    __shared__ int nstale_s;
 
     const int t = blockIdx.y, nx = gridDim.x, bx = blockIdx.x;
     const int b = 1 << lb;
@@ -97,32 +100,41 @@ ffn_gather_kernel(const WT *__restrict__ Wg, const WT *__restrict__ Wu, const WT
     const int nrows = (rows_total - bx + nx - 1) / nx;     // rows bx, bx + nx, ...
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     auto cta_sync = [] {   // the streaming warps only
-        if constexpr (FUSED) bar_sync<1, kGatherThreads>(); else __syncthreads();
+        if constexpr (SPEC) bar_sync<1, kGatherThreads>(); else __syncthreads();
     };
     pdl_launch_dependents();
-    if constexpr (FUSED) {
-        if (tid >= kGatherThreads) {   // the recovery warps
-            const int g = tid - kGatherThreads;
-            float phc[32];
-            if (fa.m <= 32) recover_load_phi<kFusedNW>(fa.Phi, fa.m, G, g, phc);
-            pdl_wait();   // y and M come from the kernel before
-            const bool writer = bx == 0;   // every CTA of the token finds the same result; one writes it
-            recover_token<kFusedNW, kFusedKC, 4>(
-                rs, g, fa.Phi, fa.gram, fa.pitch, fa.mu, fa.y + (size_t)t * fa.m, fa.m, G, k, fa.T,
-                writer && fa.support != nullptr ? fa.support + (size_t)t * k : nullptr,
-                writer && fa.z != nullptr ? fa.z + (size_t)t * k : nullptr,
-                writer && fa.resid != nullptr ? fa.resid + t : nullptr, nullptr, nullptr, writer ? status : nullptr, phc,
-                [] { __threadfence_block(); bar_arrive<2, kFusedThreads>(); },   // the streaming warps may start
-                [] { __threadfence_block(); bar_arrive<3, kFusedThreads>(); });  // the table is final
+    if constexpr (SPEC) {
+        // No wait here: the launch before this one triggered when its first slot table was in memory,
+        // and everything before THAT launch had completed by then.
+        const int32_t *table_g = support + (size_t)t * kSlotTablePitch;
+        if (tid == 0) { done_s = 0; final_s = 0; }
+        if (tid >= kGatherThreads) {   // the following warp
+            const int j = tid - kGatherThreads;
+            int g = j < k ? ld_visible(table_g + j) : 0;
+            table_s[j] = (unsigned)g < (unsigned)G ? g : 0;
+            bar_sync<2, kSpecThreads>();
+            // Keeps copying until the streaming warps have finished their pass, or the recovery has marked
+            // the table final (the mark is read first: slots read after it are the final ones).
+            for (uint32_t poll = 0; poll < kFollowLimit && *(volatile int *)&done_s == 0; ++poll) {
+                const int fin = ld_acquire(table_g + kSlotTableSlots);
+                g = j < k ? ld_visible(table_g + j) : 0;
+                table_s[j] = (unsigned)g < (unsigned)G ? g : 0;
+                if (fin != 0) {
+                    __threadfence_block();
+                    __syncwarp();
+                    if (j == 0) *(volatile int *)&final_s = 1;
+                    break;
+                }
+            }
             return;
         }
     }
     const int chunks = d / E;                                       // chunks per row
     const int nseg = (chunks + kUnitChunks * 32 - 1) / (kUnitChunks * 32);
     const int nunits = nrows * nseg;
-    pdl_wait();   // supports and activations come from the kernels before
+    if constexpr (!SPEC) pdl_wait();   // supports and activations come from the kernels before
 
-    if constexpr (!FUSED) {
+    if constexpr (!SPEC) {
         if (tid < nrows) {
             const int R = bx + nx * tid;
             // A group index outside [0, G) must not become an address: the row is read from group 0
@@ -144,8 +156,7 @@ ffn_gather_kernel(const WT *__restrict__ Wg, const WT *__restrict__ Wu, const WT
         }
         __syncthreads();
     }
-    volatile const int *table = nullptr;               // FUSED: the recovery's live slot table
-    if constexpr (FUSED) table = rs.idx;
+    volatile const int *table = table_s;               // SPEC: the slot table as the following warp last saw it
 
     uint4 *wring = ring + (size_t)warp * (kWarpRing / 16) + lane;   // this lane's column of the warp ring
     // ---- gate / up: units u = warp, warp + 16, ... ; unit u = (row u / nseg, segment u % nseg).
@@ -160,10 +171,11 @@ ffn_gather_kernel(const WT *__restrict__ Wg, const WT *__restrict__ Wu, const WT
     const WT *wg_lane = Wg + lane * E, *wu_lane = Wu + lane * E;
     const float *h_lane = h + (size_t)t * d + lane * E;
 
-    // requests the gate and up chunks of unit (r, seg) into ring stage `stage`
-    auto request_unit = [&](int r, int seg, int stage) {
+    // requests the gate and up chunks of unit (r, seg) into ring stage `stage`; settled: the final
+    // rows (chan_s) are known, otherwise (SPEC) the row's group is read from the table and remembered
+    auto request_unit = [&](int r, int seg, int stage, bool settled) {
         int chan;
-        if constexpr (FUSED) {
+        if (SPEC && !settled) {
             const int R = bx + nx * r;
             const int grp = table[R >> lb];
             if (lane == 0) ugrp_s[r][seg] = (short)grp;
@@ -183,7 +195,7 @@ ffn_gather_kernel(const WT *__restrict__ Wg, const WT *__restrict__ Wu, const WT
         }
     };
     auto issue_unit = [&](int stage) {
-        if (ci.u < nunits) request_unit(ci.r, ci.seg, stage);
+        if (ci.u < nunits) request_unit(ci.r, ci.seg, stage, false);
         cp_async_commit();  // one group per unit, empty past the end, so the wait count stays fixed
         advance(ci);
     };
@@ -220,7 +232,7 @@ ffn_gather_kernel(const WT *__restrict__ Wg, const WT *__restrict__ Wu, const WT
         return make_float2(g, up);
     };
     if (fixed_seg) load_h(cc.seg);
-    if constexpr (FUSED) bar_sync<2, kFusedThreads>();   // the table holds the first iteration's support
+    if constexpr (SPEC) bar_sync<2, kSpecThreads>();   // the table copy holds (at least) the first iterate's support
 #pragma unroll
     for (int i = 0; i < kUnitStages; ++i) issue_unit(i);
     int stage = 0;
@@ -236,27 +248,41 @@ ffn_gather_kernel(const WT *__restrict__ Wg, const WT *__restrict__ Wu, const WT
     }
     cp_async_wait<0>();
 
-    if constexpr (FUSED) {
-        bar_sync<3, kFusedThreads>();   // the recovery has finished: the table is final
+    if constexpr (SPEC) {
+        cta_sync();
+        const bool settled = *(volatile int *)&final_s != 0;   // the copy in shared memory is the final table
+        if (tid == 0) *(volatile int *)&done_s = 1;            // the following warp may leave
+        if (!settled) pdl_wait();   // else: the launch before has completed, so the table in global memory is final
         if (tid < nrows) {
             const int R = bx + nx * tid;
+            int g = settled ? table[R >> lb] : ld_visible(support + (size_t)t * kSlotTablePitch + (R >> lb));
+            if ((unsigned)g >= (unsigned)G) g = 0;   // a recovery always leaves valid groups; never an address otherwise
             bad_s[tid] = 0;
-            chan_s[tid] = (table[R >> lb] << lb) + (R & (b - 1));
+            chan_s[tid] = (g << lb) + (R & (b - 1));
         }
         cta_sync();
-        // units that were requested for a group that has since left the slot: once more, one at a time
-        // (few: the rows requested early belong to the largest entries of the first iteration)
-#pragma unroll 1
-        for (Cursor c2{warp, warp / nseg, warp % nseg}; c2.u < nunits; advance(c2)) {
-            if ((int)ugrp_s[c2.r][c2.seg] == (chan_s[c2.r] >> lb)) continue;
-            if (!fixed_seg) load_h(c2.seg);
-            request_unit(c2.r, c2.seg, 0);
-            cp_async_commit();
-            cp_async_wait<0>();
-            float2 gu = fold_unit(c2.r, c2.seg, 0);
-            gu.x = warp_sum(gu.x); gu.y = warp_sum(gu.y);
-            if (lane == 0) { red[c2.r][c2.seg][0] = gu.x; red[c2.r][c2.seg][1] = gu.y; }
+        // Units that were requested for a group that has since left its slot are fetched and folded once
+        // more.  (Few: the rows requested early belong to the largest entries of the first iterate.)  They
+        // are listed and dealt out over the warps, one per warp and round, and a round's request goes out
+        // AHEAD of the down rows, into the ring stage the down rows leave free.
+        if (tid == 0) nstale_s = 0;
+        cta_sync();
+        for (Cursor c{warp, warp / nseg, warp % nseg}; c.u < nunits; advance(c))
+            if (lane == 0 && (int)ugrp_s[c.r][c.seg] != (chan_s[c.r] >> lb)) stale_s[atomicAdd(&nstale_s, 1)] = (short)c.u;
+        cta_sync();
+    }
+    constexpr int kRedoStage = kUnitStages - 1;                       // the last unit stage = the last 8 lane slots
+    constexpr int DRS = SPEC ? (kLaneSlots - 2 * kUnitChunks) / CPT : DR;   // down rows in flight beside it
+    static_assert(DRS >= 1, "a down row must fit beside the stage kept for stale units");
+    int nstale = 0, redo_u = -1;
+    if constexpr (SPEC) {
+        nstale = nstale_s;
+        if (warp < nstale) {
+            redo_u = stale_s[warp];
+            load_h(redo_u % nseg);
+            request_unit(redo_u / nseg, redo_u % nseg, kRedoStage, true);
         }
+        cp_async_commit();
     }
 
     // ---- down rows: thread i owns chunks i, i + 512, ... of every row; lane slots of the warp ring
@@ -272,10 +298,33 @@ ffn_gather_kernel(const WT *__restrict__ Wg, const WT *__restrict__ Wu, const WT
         }
         cp_async_commit();
         ++issue_r;
-        issue_stage = issue_stage + 1 == DR ? 0 : issue_stage + 1;
+        issue_stage = issue_stage + 1 == DRS ? 0 : issue_stage + 1;
     };
 #pragma unroll 1
-    for (int r = 0; r < DR; ++r) issue_down();
+    for (int r = 0; r < DRS; ++r) issue_down();
+
+    if constexpr (SPEC) {
+        auto finish_unit = [&](int u) {
+            const int r = u / nseg, seg = u % nseg;
+            float2 gu = fold_unit(r, seg, kRedoStage);
+            gu.x = warp_sum(gu.x); gu.y = warp_sum(gu.y);
+            if (lane == 0) { red[r][seg][0] = gu.x; red[r][seg][1] = gu.y; }
+        };
+        if (redo_u >= 0) {
+            cp_async_wait<DRS>();   // the stale unit's group is older than the down rows'
+            finish_unit(redo_u);
+        }
+        // more stale units than warps (rare): the rest one at a time, each behind the down rows already in flight
+#pragma unroll 1
+        for (int i = warp + kGatherWarps; i < nstale; i += kGatherWarps) {
+            const int u = stale_s[i];
+            load_h(u % nseg);
+            request_unit(u / nseg, u % nseg, kRedoStage, true);
+            cp_async_commit();
+            cp_async_wait<0>();
+            finish_unit(u);
+        }
+    }
 
     cta_sync();
     if (tid < nrows) {
@@ -293,7 +342,7 @@ ffn_gather_kernel(const WT *__restrict__ Wg, const WT *__restrict__ Wu, const WT
     stage = 0;
 #pragma unroll 1
     for (int r = 0; r < nrows; ++r) {
-        cp_async_wait<DR - 1>();
+        cp_async_wait<DRS - 1>();
         const uint4 *src = wring + stage * (CPT * 32);
         const float a = a_s[r];
 #pragma unroll
@@ -306,9 +355,12 @@ ffn_gather_kernel(const WT *__restrict__ Wg, const WT *__restrict__ Wu, const WT
             }
         }
         issue_down();
-        stage = stage + 1 == DR ? 0 : stage + 1;
+        stage = stage + 1 == DRS ? 0 : stage + 1;
     }
     cp_async_wait<0>();
+    // SPEC: nothing is written, and this launch does not end, before the launch that runs the recovery has
+    // completed (its outputs, and the scratch the next step will reuse)
+    if constexpr (SPEC) pdl_wait();
     float *dst = partial + ((size_t)t * nx + blockIdx.x) * d + tid * E;
 #pragma unroll
     for (int j = 0; j < CPT; ++j) {
@@ -339,30 +391,27 @@ reduce_partials_kernel(const float *__restrict__ partial, int nx, int d, const f
     pdl_launch_dependents();
     pdl_wait();
     float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+    // everything this thread needs is requested in one go after the wait: the residual (first group only)
+    // and its partials p = grp, grp + 32, ..., eight at a time, added in index order
+    float4 res = make_float4(0.f, 0.f, 0.f, 0.f);
     if (col < cols) {
+        if (grp == 0 && residual != nullptr) res = ld_dep4(residual + (size_t)t * d + 4 * (size_t)col);
         const float4 *src = reinterpret_cast<const float4 *>(partial + (size_t)t * nx * d) + col;
-        // partials p = grp, grp + 32, ...: loads issued four at a time, added in index order
-        int p = grp;
-        for (; p + 3 * kReduceGroups < nx; p += 4 * kReduceGroups) {
-            const float4 v0 = ld_dep4(reinterpret_cast<const float *>(src + (size_t)p * cols)),
-                         v1 = ld_dep4(reinterpret_cast<const float *>(src + (size_t)(p + kReduceGroups) * cols)),
-                         v2 = ld_dep4(reinterpret_cast<const float *>(src + (size_t)(p + 2 * kReduceGroups) * cols)),
-                         v3 = ld_dep4(reinterpret_cast<const float *>(src + (size_t)(p + 3 * kReduceGroups) * cols));
-            s.x += v0.x; s.y += v0.y; s.z += v0.z; s.w += v0.w;
-            s.x += v1.x; s.y += v1.y; s.z += v1.z; s.w += v1.w;
-            s.x += v2.x; s.y += v2.y; s.z += v2.z; s.w += v2.w;
-            s.x += v3.x; s.y += v3.y; s.z += v3.z; s.w += v3.w;
-        }
-        for (; p < nx; p += kReduceGroups) {
-            const float4 v = ld_dep4(reinterpret_cast<const float *>(src + (size_t)p * cols));
-            s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
+        for (int p0 = grp; p0 < nx; p0 += 8 * kReduceGroups) {
+            float4 v[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int p = p0 + u * kReduceGroups;
+                v[u] = p < nx ? ld_dep4(reinterpret_cast<const float *>(src + (size_t)p * cols)) : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+#pragma unroll
+            for (int u = 0; u < 8; ++u) { s.x += v[u].x; s.y += v[u].y; s.z += v[u].z; s.w += v[u].w; }
         }
     }
     fold[grp][cl] = s;
     __syncthreads();
     if (grp == 0 && col < cols) {
-        float4 r = residual != nullptr ? ld_dep4(residual + (size_t)t * d + 4 * (size_t)col)
-                                       : make_float4(0.f, 0.f, 0.f, 0.f);
+        float4 r = res;
 #pragma unroll
         for (int g = 0; g < kReduceGroups; ++g) {
             const float4 v = fold[g][cl];
@@ -395,15 +444,15 @@ cs_status launch_check_support(cs_plan *plan, const int32_t *support, int B, cud
 }
 
 // Picks the instantiation: chunks per thread in the down phase, and whether rows need bounds checks.
-template <typename WT, bool FUSED>
+template <typename WT, bool SPEC>
 static void launch_gather_kernel(dim3 grid, cudaStream_t st, int cpt, int chunks, const WT *Wg, const WT *Wu,
                                  const WT *Wd, const float *h, const int32_t *sup, int d, int b, int k, int G,
-                                 float *partial, DeviceStatus *status, int check, const FusedArgs &fa) {
+                                 float *partial, DeviceStatus *status, int check) {
     const bool full = chunks % kGatherThreads == 0 && (cpt == 1 || cpt == 2 || cpt == 4);
     const int lb = b == 64 ? 6 : 7;
 #define CS_GATHER_CASE(N, F)                                                                              \
-    launch_pdl(true, ffn_gather_kernel<WT, N, F, FUSED>, grid, dim3(FUSED ? kFusedThreads : kGatherThreads), kRingBytes, st, \
-               Wg, Wu, Wd, h, sup, d, lb, k, G, partial, status, check, fa)
+    launch_pdl(true, ffn_gather_kernel<WT, N, F, SPEC>, grid, dim3(SPEC ? kSpecThreads : kGatherThreads), kRingBytes, st, \
+               Wg, Wu, Wd, h, sup, d, lb, k, G, partial, status, check)
     if (cpt <= 1) { if (full) CS_GATHER_CASE(1, true); else CS_GATHER_CASE(1, false); }
     else if (cpt <= 2) { if (full) CS_GATHER_CASE(2, true); else CS_GATHER_CASE(2, false); }
     else { if (full) CS_GATHER_CASE(4, true); else CS_GATHER_CASE(4, false); }
@@ -416,12 +465,11 @@ static int gather_nx(int sm_count, int nb, int rows_total, int nx_max) {
     return max(1, min(nx, min(rows_total, nx_max)));
 }
 
-// fa == NULL: supports given (`check`: validate them on the device).  Otherwise the fused step: fa holds the
-// recovery's inputs and outputs for all B tokens and `support` is unused.
+// spec: `support` is the slot table of a recovery that is still running (the small-batch step), and one SM
+// per token is left to the CTA that runs it; otherwise the supports are given (`check`: validate them).
 template <typename WT>
 static cs_status gather_typed(cs_plan *plan, const cs_layer *L, const float *h, const int32_t *support,
-                              int B, const float *residual, float *out, int check, const FusedArgs *fa,
-                              cudaStream_t st) {
+                              int B, const float *residual, float *out, int check, bool spec, cudaStream_t st) {
     const cs_config &c = plan->cfg;
     constexpr int E = Chunk<WT>::kElems;
     const int rows_total = c.k * c.group;
@@ -430,23 +478,17 @@ static cs_status gather_typed(cs_plan *plan, const cs_layer *L, const float *h, 
              *Wd = static_cast<const WT *>(L->Wd_t);
     for (int t0 = 0; t0 < B; t0 += kGatherMaxTokens) {
         const int nb = min(kGatherMaxTokens, B - t0);
-        const int nx = gather_nx(plan->sm_count, nb, rows_total, plan->nx_max);
+        const int nx = gather_nx(spec ? plan->sm_count - nb : plan->sm_count, nb, rows_total, plan->nx_max);
         dim3 grid(nx, nb);
         const float *hp = h + (size_t)t0 * c.d;
         {
             StageTimer timer(plan, CS_STAGE_EXEC, st);
-            if (fa != nullptr) {
-                FusedArgs f = *fa;
-                f.y += (size_t)t0 * c.m;
-                if (f.support != nullptr) f.support += (size_t)t0 * c.k;
-                if (f.z != nullptr) f.z += (size_t)t0 * c.k;
-                if (f.resid != nullptr) f.resid += t0;
-                launch_gather_kernel<WT, true>(grid, st, cpt, c.d / E, Wg, Wu, Wd, hp, nullptr, c.d, c.group, c.k, plan->G,
-                                               plan->partial, plan->status, 0, f);
-            } else {
+            if (spec)
+                launch_gather_kernel<WT, true>(grid, st, cpt, c.d / E, Wg, Wu, Wd, hp, support + (size_t)t0 * kSlotTablePitch,
+                                               c.d, c.group, c.k, plan->G, plan->partial, plan->status, 0);
+            else
                 launch_gather_kernel<WT, false>(grid, st, cpt, c.d / E, Wg, Wu, Wd, hp, support + (size_t)t0 * c.k, c.d,
-                                                c.group, c.k, plan->G, plan->partial, plan->status, check, FusedArgs{});
-            }
+                                                c.group, c.k, plan->G, plan->partial, plan->status, check);
         }
         plan->launches++;
         CS_CUDA_TRY(plan, cudaGetLastError());
@@ -492,24 +534,16 @@ cs_status prepare_ffn_gather(cs_plan *plan) {
 cs_status launch_ffn_gather(cs_plan *plan, const cs_layer *layer, const float *h, const int32_t *support,
                             int B, const float *residual, float *out, bool check, cudaStream_t st) {
     if (plan->cfg.w_dtype == CS_BF16)
-        return gather_typed<__nv_bfloat16>(plan, layer, h, support, B, residual, out, check, nullptr, st);
-    return gather_typed<float>(plan, layer, h, support, B, residual, out, check, nullptr, st);
+        return gather_typed<__nv_bfloat16>(plan, layer, h, support, B, residual, out, check, false, st);
+    return gather_typed<float>(plan, layer, h, support, B, residual, out, check, false, st);
 }
 
-bool fused_step_ok(const cs_plan *plan) { return plan->cfg.k <= kFusedMaxK && plan->G <= 32 * kFusedNW; }
-
-// Recovery of y (plan->gram must hold the layer's matrix: the sketch launch before formed it) and the
-// gather FFN on its result, in one launch per chunk of tokens.
-cs_status launch_recover_gather(cs_plan *plan, const cs_layer *layer, const float *h, const float *y, int B,
-                                const float *residual, float *out, int32_t *support, float *z, float *resid,
-                                cudaStream_t st) {
-    FusedArgs fa;
-    fa.Phi = layer->Phi; fa.gram = plan->gram; fa.y = y; fa.mu = layer->mu;
-    fa.m = plan->cfg.m; fa.T = plan->cfg.T; fa.pitch = gram_pitch(plan->G);
-    fa.support = support; fa.z = z; fa.resid = resid;
+// The gather FFN behind launch_sketch_recover: starts on the recovery's first slot table (plan->slot_table).
+cs_status launch_ffn_gather_spec(cs_plan *plan, const cs_layer *layer, const float *h, int B, const float *residual,
+                                 float *out, cudaStream_t st) {
     if (plan->cfg.w_dtype == CS_BF16)
-        return gather_typed<__nv_bfloat16>(plan, layer, h, nullptr, B, residual, out, 0, &fa, st);
-    return gather_typed<float>(plan, layer, h, nullptr, B, residual, out, 0, &fa, st);
+        return gather_typed<__nv_bfloat16>(plan, layer, h, plan->slot_table, B, residual, out, 0, true, st);
+    return gather_typed<float>(plan, layer, h, plan->slot_table, B, residual, out, 0, true, st);
 }
 
 
@@ -554,7 +588,7 @@ static cudaError_t static_launch(const cs_config &c, const cs_layer *L, const fl
              *Wd = static_cast<const WT *>(L->Wd_t);
     dim3 grid(nx, B);
     launch_gather_kernel<WT, false>(grid, st, cpt, c.d / E, Wg, Wu, Wd, h, support, c.d, c.group, c.k, c.d_ff / c.group,
-                                    partial, static_cast<DeviceStatus *>(nullptr), 0, FusedArgs{});
+                                    partial, static_cast<DeviceStatus *>(nullptr), 0);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     dim3 rgrid((c.d / 4 + kReduceCols - 1) / kReduceCols, B);

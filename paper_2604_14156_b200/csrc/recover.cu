@@ -26,11 +26,11 @@ recover_kernel(const float *__restrict__ Phi, const float *__restrict__ gram, fl
     float phc[32];
     if (m <= 32) recover_load_phi<NW>(Phi, m, G, g, phc);
     pdl_wait();   // y and M come from the kernel before
-    recover_token<NW, KC, 0>(s, g, Phi, gram, 32 * NW, mu, y + (size_t)t * m, m, G, k, T, support + (size_t)t * k,
+    recover_token<NW, KC, 0>(s, g, Phi, GramSource{gram, 32 * NW}, mu, y + (size_t)t * m, m, G, k, T, support + (size_t)t * k,
                              z_out != nullptr ? z_out + (size_t)t * k : nullptr,
                              resid_out != nullptr ? resid_out + t : nullptr,
                              sup0 != nullptr ? sup0 + (size_t)t * k : nullptr, z0 != nullptr ? z0 + (size_t)t * k : nullptr,
-                             status, phc, [] {}, [] {});
+                             status, phc, [] {}, [](int, int) {}, [] {});
 }
 
 typedef void (*RecoverFn)(const float *, const float *, float, const float *, int, int, int, int, int32_t *, float *, float *,

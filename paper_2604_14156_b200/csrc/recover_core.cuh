@@ -54,6 +54,7 @@ template <int NW, int KC> struct RecoverSmem {
     static constexpr int GP = 32 * NW;                 // padded number of entries = pitch of M
     static constexpr int NV = KC > 0 ? KC * 8 : GP;    // length of the iterate as the mat-vec reads it
     alignas(16) float key[GP];        // |v| of the current iterate
+    alignas(16) float red[kMaxM];     // residual r of the two-step form; partial sums of the residual norm
     alignas(16) float val[2][NV];     // the iterate, by iteration parity: slot values, or dense z
     int idx[NV];                      // list form: entry held by each slot (the support, in slot order)
     float y[kMaxM];
@@ -63,7 +64,91 @@ template <int NW, int KC> struct RecoverSmem {
     int cnt_in[4];                    // entries that entered, per warp
     int vac[4][32];                   // slots vacated by the entries that left, per warp
     int slot[GP];                     // warm start: slot of each entry, -1 outside
-    float red[kMaxM];
+};
+
+// Where the entries of M = I - mu Phi^T Phi come from.
+//   GramSource: the matrix formed by gram_rows in global memory (pitch floats per row); get(j, g) is a
+//   dependent load from L1/L2, issued only when a slot changes hands.
+//   PhiSource: no matrix at all.  Phi TRANSPOSED sits in shared memory ([G][32], rows past m zero;
+//   m <= 32) and the thread's own column of Phi in registers; get(j, g) = delta_jg - mu Phi[:, j] .
+//   Phi[:, g] is eight broadcast 16-byte reads and 32 multiply-adds, and no global load, which is what
+//   a recovery needs that runs while the rest of the GPU saturates the memory system.  The k entries
+//   of the first support are formed together with 32 * NW helper threads (PhiSource::help), which
+//   take every other slot and hand their values over through shared memory.
+struct GramSource {
+    const float *gram;
+    int pitch;
+    __device__ __forceinline__ float get(int j, int g, const float (&)[32]) const {
+        return ld_dep(gram + (size_t)j * pitch + g);
+    }
+    __device__ __forceinline__ float phi(const float *Phi, int row, int col, int G) const { return __ldg(Phi + row * G + col); }
+    // the entries of all k slots: independent loads, issued together (tid: unused)
+    template <int NR> __device__ __forceinline__ void fill(const int *idx, int k, int, int g, const float (&own)[32],
+                                                           float (&mreg)[NR]) const {
+#pragma unroll
+        for (int j = 0; j < NR; ++j)
+            if (j < k) mreg[j] = get(idx[j], g, own);
+    }
+    // the entries of the slots in `chg`: independent loads again
+    template <int NR> __device__ __forceinline__ void reload(unsigned long long chg, const int *idx, int g,
+                                                             const float (&own)[32], float (&mreg)[NR]) const {
+#pragma unroll
+        for (int j = 0; j < NR; ++j)
+            if ((chg >> j) & 1ull) mreg[j] = get(idx[j], g, own);
+    }
+};
+template <int BAR_A, int BAR_B, int THREADS> struct PhiSource {
+    const float4 *phiT_s;   // shared memory, [G][8] float4
+    float mu;
+    float *fill_s;          // shared memory, [slots][THREADS / 2]
+    __device__ __forceinline__ float get(int j, int g, const float (&own)[32]) const {
+        const float4 *col = phiT_s + j * 8;
+        float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            const float4 c = col[q];
+            a0 = fmaf(c.x, own[4 * q], a0); a1 = fmaf(c.y, own[4 * q + 1], a1);
+            a2 = fmaf(c.z, own[4 * q + 2], a2); a3 = fmaf(c.w, own[4 * q + 3], a3);
+        }
+        return (j == g ? 1.f : 0.f) - mu * ((a0 + a1) + (a2 + a3));
+    }
+    __device__ __forceinline__ float phi(const float *, int row, int col, int) const {
+        return reinterpret_cast<const float *>(phiT_s)[col * 32 + row];
+    }
+    // slots `first`, first + 2, ... for column g into the hand-over array (place tid: one per thread)
+    __device__ __forceinline__ void half(const int *idx, int k, int tid, int g, const float (&own)[32], int first) const {
+#pragma unroll 2
+        for (int j = first; j < k; j += 2) fill_s[j * (THREADS / 2) + tid] = get(idx[j], g, own);
+    }
+    template <int NR> __device__ __forceinline__ void fill(const int *idx, int k, int tid, int g, const float (&own)[32],
+                                                           float (&mreg)[NR]) const {
+        bar_sync<BAR_A, THREADS>();   // the helpers may read the table
+        half(idx, k, tid, g, own, 0);
+        __threadfence_block();
+        bar_sync<BAR_B, THREADS>();   // both halves are in the hand-over array
+#pragma unroll
+        for (int j = 0; j < NR; ++j)
+            if (j < k) mreg[j] = fill_s[j * (THREADS / 2) + tid];
+    }
+    // what helper thread tid (0 .. THREADS/2 - 1) runs, once, for a cold start with T >= 1: column g, the odd slots
+    __device__ __forceinline__ void help(const int *idx, int k, int tid, int g, const float (&own)[32]) const {
+        bar_sync<BAR_A, THREADS>();
+        half(idx, k, tid, g, own, 1);
+        __threadfence_block();
+        bar_sync<BAR_B, THREADS>();
+    }
+    // one entry per changed slot, moved into its register by a select (the slot index is the same in
+    // every thread, and changes are few): keeps the code of a support change a few hundred bytes
+    template <int NR> __device__ __forceinline__ void reload(unsigned long long chg, const int *idx, int g,
+                                                             const float (&own)[32], float (&mreg)[NR]) const {
+        while (chg != 0ull) {
+            const int js = __ffsll((long long)chg) - 1;
+            chg &= chg - 1ull;
+            const float mv = get(idx[js], g, own);
+#pragma unroll
+            for (int j = 0; j < NR; ++j) mreg[j] = j == js ? mv : mreg[j];
+        }
+    }
 };
 
 // This thread's column of Phi (needed for c): Phi is a parameter, so a caller under programmatic
@@ -76,22 +161,22 @@ __device__ __forceinline__ void recover_load_phi(const float *__restrict__ Phi, 
 }
 
 // Runs the recovery of one token.  g = this thread's entry (0 .. 32*NW-1); all 32*NW threads call it
-// together and synchronise on named barrier BAR.  pitch = floats per row of M (gram_pitch(G); the
-// dense form requires pitch == 32 * NW).  phc: the thread's column of Phi when m <= 32
+// together and synchronise on named barrier BAR.  M: where the entries of I - mu Phi^T Phi come from
+// (the dense form reads whole rows of the global matrix, whose pitch must be 32 * NW).  phc: the thread's column of Phi when m <= 32
 // (recover_load_phi), unused otherwise.  y, gram, sup0, z0 may come from the kernel before: they are
 // read with dependent loads, after the caller's wait.  table_ready() is called once by every thread
-// when the slot table s.idx first holds a support worth acting on (after the first iteration, or at
-// once when T == 0); from then on s.idx always holds k valid groups and changes only where the
-// support changes.  table_final() is called once by every thread after the last iteration, before
-// the outputs are written.
-template <int NW, int KC, int BAR, typename TableReady, typename TableFinal>
+// when the slot table s.idx first holds a support worth acting on (that of the first iterate, or the
+// start's own when T == 0 or the start is warm); from then on s.idx always holds k valid groups and changes only where the
+// support changes: slot_changed(slot, g) is called by the thread whose entry g has just taken `slot`.
+// table_final() is called once by every thread after the last iteration, before the outputs are
+// written.
+template <int NW, int KC, int BAR, typename MSource, typename TableReady, typename SlotChanged, typename TableFinal>
 __device__ __forceinline__ void recover_token(RecoverSmem<NW, KC> &s, const int g, const float *__restrict__ Phi,
-                                              const float *__restrict__ gram, const int pitch, float mu,
-                                              const float *__restrict__ y, int m, int G, int k, int T, int32_t *__restrict__ support,
+                                              const MSource M, float mu, const float *__restrict__ y, int m, int G, int k, int T, int32_t *__restrict__ support,
                                               float *__restrict__ z_out, float *__restrict__ resid_out,
                                               const int32_t *__restrict__ sup0, const float *__restrict__ z0,
                                               DeviceStatus *status, const float (&phc)[32], TableReady table_ready,
-                                              TableFinal table_final) {
+                                              SlotChanged slot_changed, TableFinal table_final) {
     constexpr int GP = 32 * NW;
     constexpr int NV = RecoverSmem<NW, KC>::NV;
     constexpr int NR = NV;                         // matrix entries a thread keeps
@@ -99,15 +184,15 @@ __device__ __forceinline__ void recover_token(RecoverSmem<NW, KC> &s, const int 
     const bool valid = g < G;
     const bool early_phi = m <= 32;
     float mreg[NR];
-    const float *mcol = gram + (valid ? g : 0);
+    const int gm = valid ? g : 0;
     if constexpr (KC > 0) {
-        // List form: the entries M[idx_j, g] that go with the list come straight from global memory (M is
-        // 30 to 60 KB and stays in L1/L2).  The first list is 0..k-1: requested at once.
+        // List form: the entries M[idx_j, g] that go with the list.  The first list (0..k-1) holds zeros
+        // unless the start is warm, and a cold first iteration hands the slots out anew: nothing to fetch yet.
 #pragma unroll
-        for (int j = 0; j < NR; ++j) mreg[j] = ld_dep(mcol + (j < k ? j : 0) * pitch);
+        for (int j = 0; j < NR; ++j) mreg[j] = 0.f;
     }
     if constexpr (KC == 0) {   // row g of M (M is symmetric: row g is the column that multiplies into entry g)
-        const float *src = gram + (size_t)(valid ? g : 0) * GP;
+        const float *src = M.gram + (size_t)gm * GP;
 #pragma unroll
         for (int j = 0; j < GP / 4; ++j) {
             const float4 q = ld_dep4(src + 4 * j);
@@ -138,7 +223,7 @@ __device__ __forceinline__ void recover_token(RecoverSmem<NW, KC> &s, const int 
     if constexpr (KC > 0) {
         if (warm) {   // the entries that go with the warm list
 #pragma unroll
-            for (int j = 0; j < NR; ++j) mreg[j] = ld_dep(mcol + s.idx[j] * pitch);
+            for (int j = 0; j < NR; ++j) mreg[j] = M.get(s.idx[j], gm, phc);
         }
     }
     // c_g = mu sum_i Phi[i,g] y_i
@@ -167,20 +252,21 @@ __device__ __forceinline__ void recover_token(RecoverSmem<NW, KC> &s, const int 
     }
     const unsigned lt_mask = (1u << lane) - 1u;
     const int rank_total = G * (G - 1) / 2;   // what the ranks of G distinct positions add up to
-    if (T == 0) table_ready();
+    if (T == 0 || warm || KC == 0) table_ready();
 
     for (int it = 0; it < T; ++it) {
-        if (it == 1) table_ready();
         const int par = it & 1;
-        // v_g = c_g + sum_j M[g, idx_j] z_j, the iterate read by broadcast
-        float a0 = cg, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+        {
+            // v_g = c_g + sum_j M[g, idx_j] z_j, the iterate read by broadcast
+            float a0 = cg, a1 = 0.f, a2 = 0.f, a3 = 0.f;
 #pragma unroll
-        for (int j = 0; j < NV / 4; ++j) {
-            const float4 zq = reinterpret_cast<const float4 *>(s.val[par])[j];
-            a0 = fmaf(mreg[4 * j], zq.x, a0); a1 = fmaf(mreg[4 * j + 1], zq.y, a1);
-            a2 = fmaf(mreg[4 * j + 2], zq.z, a2); a3 = fmaf(mreg[4 * j + 3], zq.w, a3);
+            for (int j = 0; j < NV / 4; ++j) {
+                const float4 zq = reinterpret_cast<const float4 *>(s.val[par])[j];
+                a0 = fmaf(mreg[4 * j], zq.x, a0); a1 = fmaf(mreg[4 * j + 1], zq.y, a1);
+                a2 = fmaf(mreg[4 * j + 2], zq.z, a2); a3 = fmaf(mreg[4 * j + 3], zq.w, a3);
+            }
+            v = (a0 + a1) + (a2 + a3);
         }
-        v = (a0 + a1) + (a2 + a3);
         // Keys are |v| (entries past G get -2: they precede nothing).  A NaN has no place in the order:
         // it is ranked as a zero, so that the fast test below (integer order) and the exact ranks
         // (float order) agree and every iteration still keeps exactly k entries.
@@ -200,7 +286,9 @@ __device__ __forceinline__ void recover_token(RecoverSmem<NW, KC> &s, const int 
         uint32_t gmin = 0xffffffffu, gmax = 0u;
 #pragma unroll
         for (int w = 0; w < NW; ++w) { gmin = min(gmin, s.mm[par][0][w]); gmax = max(gmax, s.mm[par][1][w]); }
-        if (gmin > gmax) continue;
+        // (a cold first iteration always takes the exact path: it hands out the slots and fetches their
+        // matrix entries)
+        if (gmin > gmax && (it > 0 || warm || KC == 0)) continue;
 
         // The support may change: exact ranks.  "a >= key" is evaluated as "a > the next float below
         // key" (-1 below zero), so that one kind of compare serves both cases.
@@ -234,60 +322,78 @@ __device__ __forceinline__ void recover_token(RecoverSmem<NW, KC> &s, const int 
             kept = kept_new;
             s.val[par ^ 1][g] = kept ? v : 0.f;
             bar_sync<BAR, GP>();
-        } else if (it == 0 && !warm) {
-            // first iteration from z = 0: no slot holds anything yet, so the slots go out by rank and
-            // the table lists the support by decreasing magnitude
-            kept = kept_new;
-            slot = rank;
-            if (kept) { s.idx[slot] = g; s.val[par ^ 1][slot] = v; }
-            bar_sync<BAR, GP>();
-#pragma unroll
-            for (int j = 0; j < NR; ++j) mreg[j] = ld_dep(mcol + s.idx[j] * pitch);
         } else {
-            // stable slots: the i-th entry that enters (by index) takes the slot of the i-th that left
-            const bool leaving = kept && !kept_new, entering = !kept && kept_new;
+            // Stable slots: the i-th entry that enters (by index) takes the slot of the i-th that left.
+            // In a cold first iteration no slot holds anything yet: every kept entry "enters", and the
+            // slots go out by rank, so that the table lists the support by decreasing magnitude.  (One
+            // code path for both on purpose: whatever runs later has then run once before anything
+            // else competes for the instruction cache's way to memory.)
+            const bool first = it == 0 && !warm;
+            const bool leaving = !first && kept && !kept_new, entering = (first || !kept) && kept_new;
             const unsigned bl = __ballot_sync(0xffffffffu, leaving), be = __ballot_sync(0xffffffffu, entering);
             if (leaving) s.vac[warp][__popc(bl & lt_mask)] = slot;
             if (lane == 0) { s.cnt[warp] = __popc(bl); s.cnt_in[warp] = __popc(be); }
             bar_sync<BAR, GP>();
             if (entering) {
-                int e = __popc(be & lt_mask);
-                for (int w = 0; w < warp; ++w) e += s.cnt_in[w];
-                int w2 = 0;
-                while (w2 < NW - 1 && e >= s.cnt[w2]) { e -= s.cnt[w2]; ++w2; }
-                // (the bound only matters for an invalid warm start, whose counts need not match)
-                slot = (int)min((unsigned)s.vac[w2][e & 31], (unsigned)(NV - 1));
+                if (first) {
+                    slot = rank;
+                } else {
+                    int e = __popc(be & lt_mask);
+                    for (int w = 0; w < warp; ++w) e += s.cnt_in[w];
+                    int w2 = 0;
+                    while (w2 < NW - 1 && e >= s.cnt[w2]) { e -= s.cnt[w2]; ++w2; }
+                    // (the bound only matters for an invalid warm start, whose counts need not match)
+                    slot = (int)min((unsigned)s.vac[w2][e & 31], (unsigned)(NV - 1));
+                }
                 s.idx[slot] = g;
+                slot_changed(slot, g);
             }
             kept = kept_new;
             if (kept) s.val[par ^ 1][slot] = v;
             unsigned long long chg = 0ull;   // slots whose entry changed
+            if (first) {
+                chg = k >= 64 ? ~0ull : (1ull << k) - 1ull;
+            } else {
 #pragma unroll
-            for (int w = 0; w < NW; ++w)
-                for (int i = 0; i < s.cnt[w]; ++i) chg |= 1ull << s.vac[w][i];
+                for (int w = 0; w < NW; ++w)
+                    for (int i = 0; i < s.cnt[w]; ++i) chg |= 1ull << s.vac[w][i];
+            }
             bar_sync<BAR, GP>();
-#pragma unroll
-            for (int j = 0; j < NR; ++j)
-                if ((chg >> j) & 1ull) mreg[j] = ld_dep(mcol + s.idx[j] * pitch);
+            if (first) table_ready();   // the table holds the first iterate's support
+            if (first) M.fill(s.idx, k, g, gm, phc, mreg);   // the entries of all k slots
+            else M.reload(chg, s.idx, gm, phc, mreg);        // those of the slots that changed hands
         }
     }
-    if (T == 1) table_ready();
     table_final();
 
-    // residual norm ||y - Phi z||_2: warp w takes rows w, w + NW, ...; lanes stride over the entries
+    // residual norm ||y - Phi z||_2
     if (resid_out != nullptr) {
-        bar_sync<BAR, GP>();
-        s.key[g] = (kept && T > 0) ? v : 0.f;   // dense z
-        bar_sync<BAR, GP>();
-        for (int row = warp; row < m; row += NW) {
-            float a = 0.f;
-#pragma unroll
-            for (int j = 0; j < NW; ++j) {
-                const int col = lane + 32 * j;
-                if (col < G) a = fmaf(__ldg(Phi + row * G + col), s.key[col], a);
+        if constexpr (KC > 0) {
+            // z has k non-zeros, held by the slots: a thread takes rows g, g + GP, ... and sums over the slots
+            // (the last iterate's values are in val[T & 1]; every path above ends on a barrier)
+            float ss = 0.f;
+            for (int row = g; row < m; row += GP) {
+                float a = 0.f;
+                for (int j = 0; j < k; ++j) a = fmaf(M.phi(Phi, row, s.idx[j], G), s.val[T & 1][j], a);
+                const float r = s.y[row] - a;
+                ss = fmaf(r, r, ss);
             }
-            a = warp_sum(a);
-            if (lane == 0) { const float r = s.y[row] - a; s.red[row] = r * r; }
+            ss = warp_sum(ss);
+            if (lane == 0) s.red[warp] = ss;
+        } else {   // dense form: warp w takes rows w, w + NW, ...; lanes stride over the entries
+            bar_sync<BAR, GP>();
+            s.key[g] = (kept && T > 0) ? v : 0.f;   // dense z
+            bar_sync<BAR, GP>();
+            for (int row = warp; row < m; row += NW) {
+                float a = 0.f;
+#pragma unroll
+                for (int j = 0; j < NW; ++j) {
+                    const int col = lane + 32 * j;
+                    if (col < G) a = fmaf(M.phi(Phi, row, col, G), s.key[col], a);
+                }
+                a = warp_sum(a);
+                if (lane == 0) { const float r = s.y[row] - a; s.red[row] = r * r; }
+            }
         }
     }
     // ascending index order: a kept entry goes to position (number of kept entries with a lower index)
@@ -307,7 +413,8 @@ __device__ __forceinline__ void recover_token(RecoverSmem<NW, KC> &s, const int 
         atomicCAS(&status->code, 0, (int)CS_ERR_NONFINITE);
     if (resid_out != nullptr && g == 0) {
         float ss = 0.f;
-        for (int row = 0; row < m; ++row) ss += s.red[row];
+        const int parts = KC > 0 ? NW : m;   // per-warp sums in the list form, per-row squares in the dense form
+        for (int i = 0; i < parts; ++i) ss += s.red[i];
         *resid_out = sqrtf(ss);
     }
 }

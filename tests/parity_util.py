@@ -36,10 +36,13 @@ def rel(a, b) -> float:
     return float(np.linalg.norm(a - b) / nb) if nb > 0 else float(np.linalg.norm(a))
 
 
-def make_plan(cfg: W.Config, max_tokens=None) -> cs.Plan:
-    return cs.Plan(cfg.d, cfg.d_ff, cfg.group, cfg.m, cfg.k, cfg.T,
+def make_plan(cfg: W.Config, max_tokens=None, speculative: bool = False) -> cs.Plan:
+    plan = cs.Plan(cfg.d, cfg.d_ff, cfg.group, cfg.m, cfg.k, cfg.T,
                    torch.float32 if cfg.w_dtype == "f32" else torch.bfloat16,
                    max_tokens or cfg.B, cfg.rms_eps)
+    if speculative:
+        plan.set_speculative(True)
+    return plan
 
 
 def device_layer(plan: cs.Plan, L: W.Layer, add_residual=None) -> cs.Layer:
