@@ -156,6 +156,85 @@ def iht(Phi, y, k: int, T: int, mu: float, z0=None) -> IHTResult:
     return IHTResult(z, sup, rh, gh[:T])
 
 
+def iht_temporal(Phi, y, k: int, T: int, mu: float, gamma: float, z_prev, z0=None) -> IHTResult:
+    """IHT on 1/2 ||y - Phi z||^2 + gamma ||z - z_prev||^2 (Sec. 5 temporal regulariser); z_prev, z0 dense [G]."""
+    Phi = _f32(Phi); y = _f64(y)
+    m, G = Phi.shape
+    z = np.empty(G); sup = np.empty(k, dtype=np.int32)
+    rh = np.empty(T + 1); gh = np.empty(max(T, 1))
+    zp = None if z_prev is None else _f64(z_prev)
+    z0a = None if z0 is None else _f64(z0)
+    lib().oracle_iht_temporal(_p(Phi), _p(y), ctypes.c_int(m), ctypes.c_int(G), ctypes.c_int(k), ctypes.c_int(T),
+                              ctypes.c_double(mu), ctypes.c_double(gamma), _p(zp), _p(z0a), _p(z), _p(sup), _p(rh), _p(gh))
+    return IHTResult(z, sup, rh, gh[:T])
+
+
+class NIHTResult(IHTResult):
+    __slots__ = ("step_hist",)
+
+
+def niht(Phi, y, k: int, T: int, mu_fallback: float) -> "NIHTResult":
+    """IHT with the normalised step mu_t = ||g_S||^2 / ||Phi g_S||^2 (no line search); see cs_oracle.c."""
+    Phi = _f32(Phi); y = _f64(y)
+    m, G = Phi.shape
+    z = np.empty(G); sup = np.empty(k, dtype=np.int32)
+    rh = np.empty(T + 1); gh = np.empty(max(T, 1)); sh = np.empty(max(T, 1))
+    lib().oracle_niht(_p(Phi), _p(y), ctypes.c_int(m), ctypes.c_int(G), ctypes.c_int(k), ctypes.c_int(T),
+                      ctypes.c_double(mu_fallback), _p(z), _p(sup), _p(rh), _p(gh), _p(sh))
+    r = NIHTResult(z, sup, rh, gh[:T])
+    r.step_hist = sh[:T]
+    return r
+
+
+class OMPResult:
+    __slots__ = ("z", "support", "order", "resid", "gap_hist")
+
+    @property
+    def min_gap(self) -> float:
+        return float(self.gap_hist.min()) if self.gap_hist.size else float("inf")
+
+
+def omp(Phi, y, k: int) -> OMPResult:
+    """Orthogonal matching pursuit over the k-subsets of the G groups; see cs_oracle.c."""
+    Phi = _f32(Phi); y = _f64(y)
+    m, G = Phi.shape
+    r = OMPResult()
+    r.z = np.empty(G); r.support = np.empty(k, dtype=np.int32); r.order = np.empty(k, dtype=np.int32)
+    r.gap_hist = np.empty(k)
+    res = ctypes.c_double(0.0)
+    lib().oracle_omp(_p(Phi), _p(y), ctypes.c_int(m), ctypes.c_int(G), ctypes.c_int(k), _p(r.z), _p(r.support),
+                     _p(r.order), ctypes.byref(res), _p(r.gap_hist))
+    r.resid = res.value
+    return r
+
+
+def srht(sign, rows, h) -> np.ndarray:
+    """Subsampled randomized Hadamard sketch of one vector [d] or a batch [B, d] (d a power of two)."""
+    sg = np.ascontiguousarray(np.asarray(sign), dtype=np.int8)
+    rw = _i32(rows); h = _f64(h)
+    d = h.shape[-1]; m = rw.shape[0]
+    assert d & (d - 1) == 0 and sg.shape == (d,)
+    flat = h.reshape(-1, d)
+    y = np.empty((flat.shape[0], m))
+    for i in range(flat.shape[0]):
+        yi = np.empty(m)
+        lib().oracle_srht(_p(sg), _p(rw), _p(np.ascontiguousarray(flat[i])), ctypes.c_int(m), ctypes.c_int(d), _p(yi))
+        y[i] = yi
+    return y.reshape(h.shape[:-1] + (m,))
+
+
+def support_drift_ratio(prev, cur) -> np.ndarray:
+    """Normalised support drift (Sec. 15 metric suite): D_t = |S_t symmetric-difference S_{t-1}| / |S_t union S_{t-1}|."""
+    a = _i32(prev); b = _i32(cur)
+    if a.ndim == 1:
+        a, b = a[None, :], b[None, :]
+    out = np.empty(a.shape[0])
+    for t in range(a.shape[0]):
+        sa, sb = set(a[t].tolist()), set(b[t].tolist())
+        out[t] = len(sa ^ sb) / len(sa | sb)
+    return out
+
+
 def ffn(W_gate, W_up, Wd_t, group: int, h, support, return_act: bool = False):
     """SwiGLU FFN of one vector h [d] restricted to the groups in ``support``."""
     wg, dt = _weights(W_gate); wu, dt2 = _weights(W_up); wd, dt3 = _weights(Wd_t)

@@ -32,6 +32,17 @@
  * Parity unpinned: nothing fixes that the support IHT returns is the *best*
  * k-subset at the benchmark shapes (IHT is a heuristic there); only
  * resid_IHT >= resid_bruteforce is asserted.
+ *
+ * Further estimators and sensors the paper names (each pinned in
+ * tests/test_oracle_solvers.py):
+ *   temporal term   (Sec. 5: Omega_temp = gamma ||alpha_t - alpha_{t-1}||^2 added to the
+ *                    recovery objective; here the projected-gradient iteration on it),
+ *   normalised step (Sec. 8 "projected proximal methods with a small fixed number of
+ *                    iterations", with the step chosen per iteration from the current
+ *                    support instead of a constant),
+ *   OMP             (Sec. 8 / Sec. 9 proposition: orthogonal matching pursuit restricted to
+ *                    the feasible supports, here any k of the G groups),
+ *   SRHT sensor     (Sec. 8: a subsampled randomized Hadamard operator as A_t).
  */
 #include <math.h>
 #include <stdint.h>
@@ -163,6 +174,218 @@ void oracle_iht(const float *Phi, const double *y, int m, int G, int k, int T, d
     for (int g = 0; g < G; ++g)
         if (keep[g]) support[c++] = g;
     free(r); free(v); free(keep);
+}
+
+/*
+ * The same estimator with the temporal regulariser of Sec. 5,
+ *     minimise  1/2 ||y - Phi z||^2 + gamma ||z - z_prev||^2   subject to  ||z||_0 <= k,
+ * by the projected-gradient step of the iteration above on this objective:
+ *     v = z + mu (Phi^T (y - Phi z) - 2 gamma (z - z_prev));   z = H_k(v).
+ * z_prev [G] is the previous decoding step's (k-sparse) estimate; gamma = 0 gives oracle_iht exactly.
+ * resid_hist records ||y - Phi z_t|| (the data term alone), as oracle_iht does.
+ */
+void oracle_iht_temporal(const float *Phi, const double *y, int m, int G, int k, int T, double mu, double gamma,
+                         const double *z_prev, const double *z0, double *z, int32_t *support,
+                         double *resid_hist, double *gap_hist) {
+    double *r = (double *)malloc(sizeof(double) * (size_t)m);
+    double *v = (double *)malloc(sizeof(double) * (size_t)G);
+    int *keep = (int *)malloc(sizeof(int) * (size_t)G);
+    for (int g = 0; g < G; ++g) z[g] = z0 ? z0[g] : 0.0;
+    oracle_hard_threshold(z, G, k, keep, NULL);
+    double rn = residual_norm(Phi, y, z, m, G, r);
+    if (resid_hist) resid_hist[0] = rn;
+    for (int t = 0; t < T; ++t) {
+        for (int g = 0; g < G; ++g) {
+            double acc = 0.0;
+            for (int i = 0; i < m; ++i) acc += (double)Phi[(size_t)i * G + g] * r[i];
+            v[g] = z[g] + mu * (acc - 2.0 * gamma * (z[g] - (z_prev ? z_prev[g] : 0.0)));
+        }
+        double gap;
+        oracle_hard_threshold(v, G, k, keep, &gap);
+        for (int g = 0; g < G; ++g) z[g] = keep[g] ? v[g] : 0.0;
+        rn = residual_norm(Phi, y, z, m, G, r);
+        if (resid_hist) resid_hist[t + 1] = rn;
+        if (gap_hist) gap_hist[t] = gap;
+    }
+    int c = 0;
+    for (int g = 0; g < G; ++g)
+        if (keep[g]) support[c++] = g;
+    free(r); free(v); free(keep);
+}
+
+/*
+ * Iterative hard thresholding with a normalised step: in every iteration the step is the one that
+ * minimises the residual along the gradient restricted to the current support S,
+ *     g = Phi^T (y - Phi z);   S = supp(z)  (for z = 0: the k entries H_k keeps of g);
+ *     mu_t = ||g_S||^2 / ||Phi g_S||^2   (mu_fallback when the denominator is 0);
+ *     z = H_k(z + mu_t g).
+ * No line search follows the step (the published method adds one for the iterations that change the
+ * support); with it left out the residual need not fall in such an iteration.
+ * step_hist [T] receives mu_t; other outputs as oracle_iht.
+ */
+void oracle_niht(const float *Phi, const double *y, int m, int G, int k, int T, double mu_fallback,
+                 double *z, int32_t *support, double *resid_hist, double *gap_hist, double *step_hist) {
+    double *r = (double *)malloc(sizeof(double) * (size_t)m);
+    double *g = (double *)malloc(sizeof(double) * (size_t)G);
+    double *v = (double *)malloc(sizeof(double) * (size_t)G);
+    int *keep = (int *)malloc(sizeof(int) * (size_t)G);
+    for (int j = 0; j < G; ++j) z[j] = 0.0;
+    oracle_hard_threshold(z, G, k, keep, NULL);
+    double rn = residual_norm(Phi, y, z, m, G, r);
+    if (resid_hist) resid_hist[0] = rn;
+    for (int t = 0; t < T; ++t) {
+        for (int j = 0; j < G; ++j) {
+            double acc = 0.0;
+            for (int i = 0; i < m; ++i) acc += (double)Phi[(size_t)i * G + j] * r[i];
+            g[j] = acc;
+        }
+        if (t == 0) oracle_hard_threshold(g, G, k, keep, NULL);   /* z = 0 has no support of its own yet */
+        double num = 0.0, den = 0.0;
+        for (int j = 0; j < G; ++j) if (keep[j]) num += g[j] * g[j];
+        for (int i = 0; i < m; ++i) {
+            double acc = 0.0;
+            for (int j = 0; j < G; ++j) if (keep[j]) acc += (double)Phi[(size_t)i * G + j] * g[j];
+            den += acc * acc;
+        }
+        double mu_t = den > 0.0 ? num / den : mu_fallback;
+        if (step_hist) step_hist[t] = mu_t;
+        for (int j = 0; j < G; ++j) v[j] = z[j] + mu_t * g[j];
+        double gap;
+        oracle_hard_threshold(v, G, k, keep, &gap);
+        for (int j = 0; j < G; ++j) z[j] = keep[j] ? v[j] : 0.0;
+        rn = residual_norm(Phi, y, z, m, G, r);
+        if (resid_hist) resid_hist[t + 1] = rn;
+        if (gap_hist) gap_hist[t] = gap;
+    }
+    int c = 0;
+    for (int j = 0; j < G; ++j)
+        if (keep[j]) support[c++] = j;
+    free(r); free(g); free(v); free(keep);
+}
+
+/*
+ * Orthogonal matching pursuit over the feasible supports (any k of the G groups): k times, pick the
+ * group whose normalised column correlates most with the residual,
+ *     j = argmax_{g not in S} |phi_g^T r| / ||phi_g||    (ties: lowest index; zero columns never),
+ * add it to S and refit  z_S = argmin ||y - Phi_S z||,  r = y - Phi_S z_S.
+ * The refit keeps an orthonormal basis Q of the chosen columns (Gram-Schmidt, applied twice) and the
+ * triangular factor R with Phi_S = Q R, so z_S = R^{-1} Q^T y by back substitution.  A column that
+ * lies in the span of those already chosen (norm after orthogonalisation <= 1e-12 of its own) adds
+ * nothing: it enters the support with coefficient 0.  If no column is left to pick (all correlations
+ * zero) the support is completed with the lowest unused indices, coefficient 0, so that exactly k
+ * indices are returned.
+ * Outputs: z [G], support [k] ascending, order [k] the groups in the order picked (-1 for
+ * completions), *resid = ||y - Phi z||, gap_hist [k] = (best - second best) / best of the normalised
+ * correlations at each pick (INFINITY when only one candidate is left, 0 for completions).
+ */
+void oracle_omp(const float *Phi, const double *y, int m, int G, int k, double *z, int32_t *support,
+                int32_t *order, double *resid, double *gap_hist) {
+    double *r = (double *)malloc(sizeof(double) * (size_t)m);
+    double *Q = (double *)calloc((size_t)m * (size_t)k, sizeof(double));      /* column s at Q[s*m ..] */
+    double *R = (double *)calloc((size_t)k * (size_t)k, sizeof(double));      /* R[a*k + s], a <= s */
+    double *qty = (double *)calloc((size_t)k, sizeof(double));
+    double *col = (double *)malloc(sizeof(double) * (size_t)m);
+    double *cn = (double *)malloc(sizeof(double) * (size_t)G);
+    int *in = (int *)calloc((size_t)G, sizeof(int));
+    int *picked = (int *)malloc(sizeof(int) * (size_t)k);
+    int *live = (int *)calloc((size_t)k, sizeof(int));                        /* basis vector exists for pick s */
+    for (int i = 0; i < m; ++i) r[i] = y[i];
+    for (int g = 0; g < G; ++g) {
+        double ss = 0.0;
+        for (int i = 0; i < m; ++i) ss += (double)Phi[(size_t)i * G + g] * (double)Phi[(size_t)i * G + g];
+        cn[g] = sqrt(ss);
+        z[g] = 0.0;
+    }
+    int ns = 0;
+    for (int s = 0; s < k; ++s) {
+        int best = -1, cand = 0;
+        double bv = 0.0, second = 0.0;
+        for (int g = 0; g < G; ++g) {
+            if (in[g] || cn[g] == 0.0) continue;
+            double acc = 0.0;
+            for (int i = 0; i < m; ++i) acc += (double)Phi[(size_t)i * G + g] * r[i];
+            double c = fabs(acc) / cn[g];
+            ++cand;
+            if (c > bv) { second = bv; bv = c; best = g; }
+            else if (c > second) second = c;
+        }
+        if (best < 0 || bv == 0.0) {          /* nothing correlates: complete with the lowest unused indices */
+            int g = 0;
+            while (in[g]) ++g;
+            in[g] = 1; picked[s] = g; order[s] = -1;
+            if (gap_hist) gap_hist[s] = 0.0;
+            ++ns;
+            continue;
+        }
+        if (gap_hist) gap_hist[s] = cand > 1 ? (bv - second) / bv : INFINITY;
+        in[best] = 1; picked[s] = best; order[s] = best; ++ns;
+        for (int i = 0; i < m; ++i) col[i] = (double)Phi[(size_t)i * G + best];
+        for (int pass = 0; pass < 2; ++pass)          /* Gram-Schmidt, twice */
+            for (int a = 0; a < s; ++a) {
+                if (!live[a]) continue;
+                double dot = 0.0;
+                for (int i = 0; i < m; ++i) dot += Q[(size_t)a * m + i] * col[i];
+                for (int i = 0; i < m; ++i) col[i] -= dot * Q[(size_t)a * m + i];
+                R[(size_t)a * k + s] += dot;
+            }
+        double nn = 0.0;
+        for (int i = 0; i < m; ++i) nn += col[i] * col[i];
+        nn = sqrt(nn);
+        if (nn <= 1e-12 * cn[best]) continue;          /* in the span already: coefficient stays 0 */
+        live[s] = 1;
+        R[(size_t)s * k + s] = nn;
+        double qy = 0.0;
+        for (int i = 0; i < m; ++i) { Q[(size_t)s * m + i] = col[i] / nn; qy += Q[(size_t)s * m + i] * y[i]; }
+        qty[s] = qy;
+        /* r = y - Q Q^T y over the live basis vectors */
+        for (int i = 0; i < m; ++i) r[i] = y[i];
+        for (int a = 0; a <= s; ++a) {
+            if (!live[a]) continue;
+            for (int i = 0; i < m; ++i) r[i] -= qty[a] * Q[(size_t)a * m + i];
+        }
+    }
+    /* z_S = R^{-1} Q^T y by back substitution over the live picks */
+    double *coef = (double *)calloc((size_t)k, sizeof(double));
+    for (int s = ns - 1; s >= 0; --s) {
+        if (!live[s]) continue;
+        double acc = qty[s];
+        for (int b = s + 1; b < ns; ++b)
+            if (live[b]) acc -= R[(size_t)s * k + b] * coef[b];
+        coef[s] = acc / R[(size_t)s * k + s];
+    }
+    for (int s = 0; s < ns; ++s) z[picked[s]] = coef[s];
+    int c = 0;
+    for (int g = 0; g < G; ++g)
+        if (in[g]) support[c++] = g;
+    double ss = 0.0;
+    for (int i = 0; i < m; ++i) {
+        double acc = 0.0;
+        for (int g = 0; g < G; ++g) acc += (double)Phi[(size_t)i * G + g] * z[g];
+        ss += (y[i] - acc) * (y[i] - acc);
+    }
+    if (resid) *resid = sqrt(ss);
+    free(r); free(Q); free(R); free(qty); free(col); free(cn); free(in); free(picked); free(live); free(coef);
+}
+
+/*
+ * Sensor, structured: a subsampled randomized Hadamard operator (Sec. 8),
+ *     y_r = (1 / sqrt(m)) sum_i H[rows[r], i] sign[i] h[i],   H[a, i] = (-1)^popcount(a & i),
+ * with d a power of two, sign[i] in {+1, -1} and rows [m] distinct indices in [0, d).  Written out
+ * term by term (no fast transform): m * d multiply-adds.
+ */
+void oracle_srht(const int8_t *sign, const int32_t *rows, const double *h, int m, int d, double *y) {
+    double scale = 1.0 / sqrt((double)m);
+    for (int r = 0; r < m; ++r) {
+        double acc = 0.0;
+        unsigned a = (unsigned)rows[r];
+        for (int i = 0; i < d; ++i) {
+            unsigned bits = a & (unsigned)i, par = 0;
+            while (bits) { par ^= 1u; bits &= bits - 1u; }
+            double term = (double)sign[i] * h[i];
+            acc += par ? -term : term;
+        }
+        y[r] = scale * acc;
+    }
 }
 
 static double silu(double x) { return x / (1.0 + exp(-x)); }

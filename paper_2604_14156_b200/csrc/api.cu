@@ -245,11 +245,24 @@ static cs_status exec_dispatch(cs_plan *plan, const cs_layer *layer, const float
         cs_status s = launch_check_support(plan, support, B, st);
         if (s != CS_OK) return s;
     }
-    if (use_decode_mma(plan, B))
-        return exec_decode_overlapped(plan, layer, h, B, residual, out, st,
-                                      [&](cudaStream_t side) { return launch_bucket(plan, support, B, side); });
     __nv_bfloat16 *x_hi = static_cast<__nv_bfloat16 *>(plan->x_bf16);
     __nv_bfloat16 *x_lo = x_hi + (size_t)plan->cfg.max_tokens * plan->cfg.d;
+    if (use_decode_mma(plan, B)) {
+        // The supports are known before the GEMMs here.  While the batch is small enough that a fair share
+        // of the groups is in nobody's support (expected unused fraction (1 - k/G)^B of about 8 % or more),
+        // the buckets are formed first and gate/up runs over the union list only, with the membership masks
+        // applied in its epilogue; beyond that the union is (nearly) every group and bucketing runs beside
+        // the dense gate/up GEMM instead.
+        if (2 * B * plan->cfg.k <= 5 * plan->G) {
+            cs_status s = launch_bucket(plan, support, B, st);
+            if (s == CS_OK) s = launch_split_bf16(plan, h, x_hi, x_lo, (size_t)B * plan->cfg.d, st);
+            if (s == CS_OK) s = launch_decode_gateup(plan, layer, x_hi, x_lo, B, true, st);
+            if (s == CS_OK) s = launch_decode_down(plan, layer, B, false, residual, out, st);
+            return s;
+        }
+        return exec_decode_overlapped(plan, layer, h, B, residual, out, st,
+                                      [&](cudaStream_t side) { return launch_bucket(plan, support, B, side); });
+    }
     cs_status s = launch_split_bf16(plan, h, x_hi, x_lo, (size_t)B * plan->cfg.d, st);
     if (s != CS_OK) return s;
     s = launch_bucket(plan, support, B, st);
