@@ -341,6 +341,8 @@ def bench_decode(cfg, args, K, Wm, rank, world, local, dev, primary):
                      "frac_of_8tbs_nominal": ab["total"] / (step_us * 1e-6) / 1e9 / 8000.0,
                      "union_groups": union, "groups_streamed": (cfg.G if mma else union)},
     }
+    if primary and rank == 0:
+        out["planted_recovery"] = planted_recovery(cfg, dev)
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         cpu_layers = [L.to("cpu") for L in layers_raw[:2]]
         out["cpu_baseline"] = cpu_baseline(cfg, cpu_layers, hx, seconds=10.0 if primary else 3.0, single=primary)
@@ -442,6 +444,34 @@ def bench_prompt(cfg, args, K, Wm, rank, world, local, dev, primary):
         res["cpu_baseline"] = cpu_baseline_prompt(cfg, raw[0].to("cpu"), Hs[0].cpu(), seconds=10.0 if primary else 3.0)
     plan.close()
     return res
+
+
+def planted_recovery(cfg, dev, trials: int = 256):
+    """How often each estimator returns a planted support (noiseless, |c| >= 0.5) at this workload's m and G,
+    for sparsity levels from easy to the workload's own k: the library's kernels through cs_recover_ex."""
+    import numpy as np
+    import paper_2604_14156_b200 as cs
+    from gen import rng
+    out = {}
+    Phi = rng.normal(cfg.seed, (W.T_PHI, 0), (cfg.m, cfg.G), dtype=torch.float32, scale=cfg.m ** -0.5)
+    mu = W.spectral_step(Phi)
+    Pn = Phi.double()
+    for k in sorted({max(1, cfg.k // 8), max(1, cfg.k // 4), max(1, cfg.k // 2), cfg.k}):
+        plan = cs.Plan(cfg.d, cfg.d_ff, cfg.group, cfg.m, k, 40, torch.float32 if cfg.w_dtype == "f32" else torch.bfloat16,
+                       trials, cfg.rms_eps)
+        sup = rng.k_subset(cfg.seed, (97, k), cfg.G, k, rows=trials)
+        c = rng.normal(cfg.seed, (98, k), (trials, k))
+        c = torch.sign(c) * c.abs().clamp_min(0.5)
+        y = torch.einsum("tk,tmk->tm", c, Pn[:, sup.long()].permute(1, 0, 2)).float().to(dev)
+        row = {}
+        for solver in ("iht", "niht", "omp"):
+            if solver == "omp" and k > 64:
+                continue
+            got, _, _ = cs.cs_recover_ex(plan, Phi.to(dev), mu, y, cs.StepOptions(plan, trials, solver=solver, device=dev))
+            row[solver] = float((got.cpu() == sup).all(dim=1).float().mean())
+        out[f"k={k}"] = row
+        plan.close()
+    return {"m": cfg.m, "G": cfg.G, "trials": trials, "iterations": 40, "rate_by_sparsity": out}
 
 
 def cpu_baseline(cfg, cpu_layers, hx, seconds: float, single: bool):

@@ -125,6 +125,63 @@ cs_status cs_support_drift(cs_plan *plan, const int32_t *support_prev, const int
                            int32_t *drift, void *stream);
 
 /*
+ * Normalised support drift between consecutive decoding steps (Sec. 15 metric suite):
+ *     D[t] = |S_t symmetric-difference S_{t-1}| / |S_t union S_{t-1}|,
+ * 0 for identical supports, 1 for disjoint ones.  Arguments as cs_support_drift; `delta` (the count of
+ * cs_support_drift) and `D` may each be NULL.
+ */
+cs_status cs_support_drift_ratio(cs_plan *plan, const int32_t *support_prev, const int32_t *support_cur, int32_t B,
+                                 int32_t *delta, float *D, void *stream);
+
+/*
+ * Options of one estimation / one step (cs_recover_ex, cs_layer_step_ex).  A zero-filled struct with
+ * T = -1 asks for exactly what cs_recover / cs_layer_step do.  HOST memory, read before the call returns;
+ * the pointers inside are DEVICE pointers.
+ */
+typedef enum {
+    CS_SOLVER_IHT = 0,   /* fixed step mu (cs_recover) */
+    CS_SOLVER_NIHT = 1,  /* the step of every iteration chosen from the current support S:
+                            mu_t = ||g_S||^2 / ||Phi g_S||^2, g = Phi^T (y - Phi z)  (Sec. 8: a projected method with
+                            a small fixed number of iterations; no line search follows the step).  `mu` is only
+                            the fallback when the denominator vanishes. */
+    CS_SOLVER_OMP = 2    /* orthogonal matching pursuit over the feasible supports, any k of the G groups (Sec. 8;
+                            Sec. 9 incoherence proposition): k picks by normalised correlation with the residual
+                            (ties: lowest index), each followed by the least-squares refit.  Needs k <= 64. */
+} cs_solver;
+
+typedef struct {
+    int32_t solver;              /* cs_solver */
+    int32_t T;                   /* iterations of CS_SOLVER_IHT / NIHT for this call; < 0: the plan's */
+    const int32_t *support_prev; /* [B,k] supports of the previous decoding step (ascending, distinct), or NULL */
+    const float *z_prev;         /* [B,k] its coefficients (needed with support_prev unless only drift is asked) */
+    int32_t warm_start;          /* CS_SOLVER_IHT: start from (support_prev, z_prev) instead of 0 (Sec. 8 warm start) */
+    float gamma;                 /* CS_SOLVER_IHT: weight of the temporal regulariser gamma ||z - z_prev||^2 (Sec. 5);
+                                    the step becomes  v = z + mu (Phi^T (y - Phi z) - 2 gamma (z - z_prev)).  0: none */
+    int32_t reuse_support;       /* cs_layer_step_ex: skip sensing and recovery and execute on support_prev
+                                    (Sec. 5: "updated every step, every few steps, or event-triggered") */
+    const uint32_t *srht_sign;   /* cs_layer_step_ex: sense with the subsampled randomized Hadamard operator */
+    const int32_t *srht_rows;    /*   (cs_sketch_srht) instead of layer->S; both NULL: the dense sketch */
+    int32_t *delta_out;          /* [B] |S_t symmetric-difference S_{t-1}| against support_prev, or NULL */
+    float *drift_out;            /* [B] the normalised drift D_t, or NULL */
+} cs_step_options;
+
+/* The estimator with options: solver, iteration count, warm start, temporal term.  Outputs as cs_recover. */
+cs_status cs_recover_ex(cs_plan *plan, const float *Phi, float mu, const float *y, int32_t B,
+                        const cs_step_options *opt, int32_t *support, float *z, float *resid, void *stream);
+
+/*
+ * Structured sensor (Sec. 8: "subsampled randomized Hadamard operators when implementation efficiency is
+ * important"):  y[t, r] = (1/sqrt(m)) sum_i H[rows[r], i] s_i h[t, i],  H[a, i] = (-1)^popcount(a & i), s_i = -1
+ * where bit i of sign_bits is set (bit i of word i / 32), else +1.  The fast transform costs d log2 d additions
+ * and reads d / 8 + 4 m bytes of operator instead of the 4 m d bytes of a dense S.
+ *   sign_bits [d/32] uint32, rows [m] int32 distinct in [0, d), h [B,d] f32 -> y [B,m] f32.
+ * d must be a power of two between 256 and 8192 (CS_ERR_UNSUPPORTED otherwise).  The recovery that follows
+ * uses Phi = (this operator) * Psi, which the caller precomputes as it precomputes S = Phi * A for the dense one.
+ */
+cs_status cs_sketch_srht(cs_plan *plan, const uint32_t *sign_bits, const int32_t *rows, const float *h, int32_t B,
+                         float *y, void *stream);
+
+/*
  * Uncertainty-driven sensing controller (Sec. 8.1): per token, the predictive entropy of the
  * previous decoding step's distribution over the vocabulary and the measurement budget for the
  * current step,
@@ -217,6 +274,34 @@ cs_status cs_ffn_exec_static(const cs_config *cfg, const cs_layer *layer, const 
  */
 cs_status cs_layer_step(cs_plan *plan, const cs_layer *layer, const float *x, int32_t B, float *x_out,
                         int32_t *support_out, float *z_out, float *resid_out, void *stream);
+
+/*
+ * cs_layer_step with options (opt == NULL: cs_layer_step itself): another estimator, a warm start and
+ * the temporal term from the previous step's result, the structured sensor, the drift against the
+ * previous supports, or no estimation at all (reuse_support).  The stages run one after the other on
+ * `stream` (the overlap of cs_layer_step's default path is not used).  With srht_sign / srht_rows the
+ * layer must have no RMSNorm (rms_gamma == NULL) and layer->S is not read.
+ */
+cs_status cs_layer_step_ex(cs_plan *plan, const cs_layer *layer, const float *x, int32_t B,
+                           const cs_step_options *opt, float *x_out, int32_t *support_out, float *z_out,
+                           float *resid_out, void *stream);
+
+/*
+ * Confidence fallback (Sec. 12, online phase: when "the recovery confidence falls below a threshold, the
+ * system may revert temporarily to a denser support").  Runs cs_layer_step_ex on `plan`; a token whose
+ * relative residual ||y - Phi z_T|| / ||y|| exceeds `tau` is not trusted, and the step is run again for
+ * those tokens alone on `dense`, a plan of the same layer shape with a larger k (k = G: the dense FFN),
+ * whose outputs replace theirs in x_out.
+ *   flags_out [B] int32 (device; 1 = fell back) may be NULL; *n_fallback (HOST) receives their number.
+ *   support_out / z_out / resid_out describe the FIRST recovery of every token (a token that fell back
+ *   executed on the k_dense groups its second recovery kept, which are not returned).
+ * THIS CALL SYNCHRONISES `stream` once (the number of low-confidence tokens decides what is launched
+ * next), so it cannot be captured in a graph; opt->reuse_support must be 0.
+ */
+cs_status cs_layer_step_fallback(cs_plan *plan, cs_plan *dense, const cs_layer *layer, const float *x, int32_t B,
+                                 const cs_step_options *opt, float tau, float *x_out, int32_t *support_out,
+                                 float *z_out, float *resid_out, int32_t *flags_out, int32_t *n_fallback,
+                                 void *stream);
 
 /*
  * Prompt-level support (Sec. 4): one support for the whole prompt from the mean prompt sketch,

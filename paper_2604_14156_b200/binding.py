@@ -29,6 +29,16 @@ class _Config(ctypes.Structure):
                 ("w_dtype", ctypes.c_int32), ("max_tokens", ctypes.c_int32), ("rms_eps", ctypes.c_float)]
 
 
+class _StepOptions(ctypes.Structure):
+    _fields_ = [("solver", ctypes.c_int32), ("T", ctypes.c_int32), ("support_prev", ctypes.c_void_p),
+                ("z_prev", ctypes.c_void_p), ("warm_start", ctypes.c_int32), ("gamma", ctypes.c_float),
+                ("reuse_support", ctypes.c_int32), ("srht_sign", ctypes.c_void_p), ("srht_rows", ctypes.c_void_p),
+                ("delta_out", ctypes.c_void_p), ("drift_out", ctypes.c_void_p)]
+
+
+SOLVERS = {"iht": 0, "niht": 1, "omp": 2}
+
+
 class _Layer(ctypes.Structure):
     _fields_ = [("S", ctypes.c_void_p), ("Phi", ctypes.c_void_p), ("W_gate", ctypes.c_void_p),
                 ("W_up", ctypes.c_void_p), ("Wd_t", ctypes.c_void_p), ("rms_gamma", ctypes.c_void_p),
@@ -78,6 +88,14 @@ def load_library():
     lib.cs_plan_crossover.argtypes = [vp]
     lib.cs_plan_crossover.restype = ctypes.c_int32
     lib.cs_plan_stage_times.argtypes = [vp, vp, ctypes.POINTER(f32 * 5)]
+    lib.cs_support_drift_ratio.argtypes = [vp, vp, vp, i32, vp, vp, vp]
+    lib.cs_recover_ex.argtypes = [vp, vp, f32, vp, i32, ctypes.POINTER(_StepOptions), vp, vp, vp, vp]
+    lib.cs_sketch_srht.argtypes = [vp, vp, vp, vp, i32, vp, vp]
+    lib.cs_layer_step_ex.argtypes = [vp, ctypes.POINTER(_Layer), vp, i32, ctypes.POINTER(_StepOptions), vp, vp, vp, vp, vp]
+    lib.cs_layer_step_fallback.argtypes = [vp, vp, ctypes.POINTER(_Layer), vp, i32, ctypes.POINTER(_StepOptions), f32, vp,
+                                           vp, vp, vp, vp, ctypes.POINTER(i32), vp]
+    for name in ("cs_support_drift_ratio", "cs_recover_ex", "cs_sketch_srht", "cs_layer_step_ex", "cs_layer_step_fallback"):
+        getattr(lib, name).restype = ctypes.c_int
     lib.cs_ffn_exec_static.argtypes = [ctypes.POINTER(_Config), ctypes.POINTER(_Layer), vp, vp, i32, vp, vp, vp]
     lib.cs_ffn_exec_static.restype = ctypes.c_int
     lib.cs_bucket.argtypes = [vp, vp, i32, vp, vp, vp, vp]
@@ -248,6 +266,93 @@ def cs_support_drift(plan: Plan, support_prev, support_cur, stream=None):
                                          _ptr(support_cur, torch.int32, "support_cur", (B, plan.k)), B,
                                          drift.data_ptr(), _stream(stream)), "cs_support_drift")
     return drift
+
+
+def cs_support_drift_ratio(plan: Plan, support_prev, support_cur, stream=None):
+    """(Delta_t [B] int32, D_t [B] float32): the drift count and the normalised drift of Sec. 15."""
+    B = support_cur.shape[0]
+    delta = torch.empty((B,), dtype=torch.int32, device=support_cur.device)
+    D = torch.empty((B,), dtype=torch.float32, device=support_cur.device)
+    plan.check(plan.lib.cs_support_drift_ratio(plan.handle, _ptr(support_prev, torch.int32, "support_prev", (B, plan.k)),
+                                               _ptr(support_cur, torch.int32, "support_cur", (B, plan.k)), B,
+                                               delta.data_ptr(), D.data_ptr(), _stream(stream)), "cs_support_drift_ratio")
+    return delta, D
+
+
+class StepOptions:
+    """Options of cs_recover_ex / cs_layer_step_ex; keeps the tensors it points at alive."""
+
+    def __init__(self, plan: Plan, B: int, solver: str = "iht", T: int = -1, support_prev=None, z_prev=None,
+                 warm_start: bool = False, gamma: float = 0.0, reuse_support: bool = False, srht=None,
+                 want_drift: bool = False, device="cuda"):
+        self.delta = self.drift = None
+        if want_drift:
+            self.delta = torch.empty((B,), dtype=torch.int32, device=device)
+            self.drift = torch.empty((B,), dtype=torch.float32, device=device)
+        self.keep = (support_prev, z_prev, srht)
+        sign, rows = (None, None) if srht is None else srht
+        self.c = _StepOptions(
+            SOLVERS[solver], int(T), _ptr(support_prev, torch.int32, "support_prev", (B, plan.k)),
+            _ptr(z_prev, torch.float32, "z_prev", (B, plan.k)), int(bool(warm_start)), float(gamma),
+            int(bool(reuse_support)), _ptr(sign, torch.int32, "srht sign bits", (plan.d // 32,)),
+            _ptr(rows, torch.int32, "srht rows", (plan.m,)),
+            None if self.delta is None else self.delta.data_ptr(), None if self.drift is None else self.drift.data_ptr())
+
+
+def cs_recover_ex(plan: Plan, Phi, mu: float, y, options: StepOptions, stream=None):
+    B = y.shape[0]
+    dev = y.device
+    support = torch.empty((B, plan.k), dtype=torch.int32, device=dev)
+    z = torch.empty((B, plan.k), dtype=torch.float32, device=dev)
+    resid = torch.empty((B,), dtype=torch.float32, device=dev)
+    plan.check(plan.lib.cs_recover_ex(plan.handle, _ptr(Phi, torch.float32, "Phi", (plan.m, plan.G)), float(mu),
+                                      _ptr(y, torch.float32, "y", (B, plan.m)), B, ctypes.byref(options.c),
+                                      support.data_ptr(), z.data_ptr(), resid.data_ptr(), _stream(stream)), "cs_recover_ex")
+    return support, z, resid
+
+
+def cs_sketch_srht(plan: Plan, sign_bits, rows, h, stream=None):
+    """y [B, m] of the subsampled randomized Hadamard sketch; sign_bits [d/32] int32 (bit i set: s_i = -1), rows [m] int32."""
+    B = h.shape[0]
+    y = torch.empty((B, plan.m), dtype=torch.float32, device=h.device)
+    plan.check(plan.lib.cs_sketch_srht(plan.handle, _ptr(sign_bits, torch.int32, "sign_bits", (plan.d // 32,)),
+                                       _ptr(rows, torch.int32, "rows", (plan.m,)), _ptr(h, torch.float32, "h", (B, plan.d)),
+                                       B, y.data_ptr(), _stream(stream)), "cs_sketch_srht")
+    return y
+
+
+def cs_layer_step_ex(plan: Plan, layer: Layer, x, options: StepOptions, x_out=None, stream=None):
+    """Returns (x_out, support, z, resid)."""
+    B = x.shape[0]
+    dev = x.device
+    x_out = torch.empty_like(x) if x_out is None else x_out
+    support = torch.empty((B, plan.k), dtype=torch.int32, device=dev)
+    z = torch.zeros((B, plan.k), dtype=torch.float32, device=dev)
+    resid = torch.zeros((B,), dtype=torch.float32, device=dev)
+    plan.check(plan.lib.cs_layer_step_ex(plan.handle, ctypes.byref(layer.c), _ptr(x, torch.float32, "x", (B, plan.d)), B,
+                                         ctypes.byref(options.c), _ptr(x_out, torch.float32, "x_out", (B, plan.d)),
+                                         support.data_ptr(), z.data_ptr(), resid.data_ptr(), _stream(stream)),
+               "cs_layer_step_ex")
+    return x_out, support, z, resid
+
+
+def cs_layer_step_fallback(plan: Plan, dense: Plan, layer: Layer, x, tau: float, options: Optional[StepOptions] = None,
+                           stream=None):
+    """Returns (x_out, support, z, resid, flags, n_fallback); synchronises the stream (see include/cs.h)."""
+    B = x.shape[0]
+    dev = x.device
+    x_out = torch.empty_like(x)
+    support = torch.empty((B, plan.k), dtype=torch.int32, device=dev)
+    z = torch.empty((B, plan.k), dtype=torch.float32, device=dev)
+    resid = torch.empty((B,), dtype=torch.float32, device=dev)
+    flags = torch.empty((B,), dtype=torch.int32, device=dev)
+    n = ctypes.c_int32(0)
+    plan.check(plan.lib.cs_layer_step_fallback(plan.handle, dense.handle, ctypes.byref(layer.c),
+                                               _ptr(x, torch.float32, "x", (B, plan.d)), B,
+                                               None if options is None else ctypes.byref(options.c), float(tau),
+                                               x_out.data_ptr(), support.data_ptr(), z.data_ptr(), resid.data_ptr(),
+                                               flags.data_ptr(), ctypes.byref(n), _stream(stream)), "cs_layer_step_fallback")
+    return x_out, support, z, resid, flags, n.value
 
 
 def cs_uds_budget(plan: Plan, logits, m_base: float, gamma: float, m_min: int, m_max: int, stream=None):

@@ -84,6 +84,10 @@ cs_status cs_plan_create(const cs_config *cfg, cs_plan **out) {
     alloc((void **)&p->sup_buf, nt * cfg->k * sizeof(int32_t));
     alloc((void **)&p->partial, (size_t)kGatherMaxTokens * p->nx_max * cfg->d * sizeof(float));
     alloc((void **)&p->gram, (size_t)kMaxG * kMaxG * sizeof(float));
+    alloc((void **)&p->resid_buf, nt * sizeof(float));
+    alloc((void **)&p->fb_flags, nt * sizeof(int32_t));
+    alloc((void **)&p->fb_list, nt * sizeof(int32_t));
+    alloc((void **)&p->fb_count, sizeof(int32_t));
     alloc((void **)&p->slot_table, nt * kSlotTablePitch * sizeof(int32_t));
     alloc((void **)&p->ticket, nt * sizeof(unsigned));
     alloc((void **)&p->hbar, (size_t)cfg->d * sizeof(float));
@@ -121,6 +125,7 @@ cs_status cs_plan_create(const cs_config *cfg, cs_plan **out) {
     if (e == cudaSuccess) e = cudaMemset(p->ticket, 0, nt * sizeof(unsigned));
     if (e == cudaSuccess) e = cudaMemset(p->slot_table, 0, nt * kSlotTablePitch * sizeof(int32_t));
     if (e == cudaSuccess && prepare_sketch(p) != CS_OK) e = cudaErrorUnknown;
+    if (e == cudaSuccess && prepare_solvers(p) != CS_OK) e = cudaErrorUnknown;
     if (e == cudaSuccess && prepare_ffn_gather(p) != CS_OK) e = cudaErrorUnknown;
     if (e == cudaSuccess && p->mma_ok && prepare_ffn_mma(p) != CS_OK) e = cudaErrorUnknown;
     if (e != cudaSuccess) {
@@ -134,7 +139,8 @@ cs_status cs_plan_create(const cs_config *cfg, cs_plan **out) {
 cs_status cs_plan_destroy(cs_plan *p) {
     if (p == nullptr) return CS_ERR_NULL;
     cudaFree(p->n_buf); cudaFree(p->y_buf); cudaFree(p->sup_buf);
-    cudaFree(p->partial); cudaFree(p->gram); cudaFree(p->slot_table); cudaFree(p->ticket); cudaFree(p->hbar); cudaFree(p->colsum);
+    cudaFree(p->partial); cudaFree(p->gram); cudaFree(p->slot_table); cudaFree(p->ticket);
+    cudaFree(p->resid_buf); cudaFree(p->fb_flags); cudaFree(p->fb_list); cudaFree(p->fb_count); cudaFree(p->hbar); cudaFree(p->colsum);
     cudaFree(p->status); cudaFree(p->x_host_in); cudaFree(p->x_host_out);
     cudaFree(p->mask); cudaFree(p->gmask); cudaFree(p->counts); cudaFree(p->offsets); cudaFree(p->token_ids); cudaFree(p->glist);
     cudaFree(p->nu); cudaFree(p->x_bf16); cudaFree(p->act); cudaFree(p->mma_partial);
@@ -183,7 +189,71 @@ cs_status cs_support_drift(cs_plan *plan, const int32_t *support_prev, const int
     cs_status s = launch_check_support(plan, support_prev, B, st);
     if (s == CS_OK) s = launch_check_support(plan, support_cur, B, st);
     if (s != CS_OK) return s;
-    return launch_support_drift(plan, support_prev, support_cur, B, drift, st);
+    return launch_support_drift(plan, support_prev, support_cur, B, drift, nullptr, st);
+}
+
+cs_status cs_support_drift_ratio(cs_plan *plan, const int32_t *support_prev, const int32_t *support_cur, int32_t B,
+                                 int32_t *delta, float *D, void *stream) {
+    if (plan == nullptr || support_prev == nullptr || support_cur == nullptr || (delta == nullptr && D == nullptr))
+        return CS_ERR_NULL;
+    if (B <= 0 || B > plan->cfg.max_tokens) return CS_ERR_SHAPE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cs_status s = launch_check_support(plan, support_prev, B, st);
+    if (s == CS_OK) s = launch_check_support(plan, support_cur, B, st);
+    if (s != CS_OK) return s;
+    return launch_support_drift(plan, support_prev, support_cur, B, delta, D, st);
+}
+
+static cs_status check_options(const cs_plan *plan, const cs_step_options *o, bool step) {
+    if (o->solver != CS_SOLVER_IHT && o->solver != CS_SOLVER_NIHT && o->solver != CS_SOLVER_OMP) return CS_ERR_UNSUPPORTED;
+    if (o->solver == CS_SOLVER_OMP && plan->cfg.k > 64) return CS_ERR_UNSUPPORTED;
+    if (!isfinite(o->gamma) || o->gamma < 0.f) return CS_ERR_NONFINITE;
+    const bool needs_prev = o->warm_start || o->gamma > 0.f;
+    if (needs_prev && (o->support_prev == nullptr || o->z_prev == nullptr)) return CS_ERR_NULL;
+    if ((o->delta_out != nullptr || o->drift_out != nullptr || (step && o->reuse_support)) && o->support_prev == nullptr)
+        return CS_ERR_NULL;
+    if ((o->warm_start || o->gamma > 0.f) && o->solver != CS_SOLVER_IHT) return CS_ERR_UNSUPPORTED;
+    if (o->warm_start && o->T == 0) return CS_ERR_SHAPE;
+    if ((o->srht_sign == nullptr) != (o->srht_rows == nullptr)) return CS_ERR_NULL;
+    return CS_OK;
+}
+
+// The estimator an options struct asks for, on y; gram_ready: plan->gram holds this Phi's matrix.
+static cs_status recover_with(cs_plan *plan, const float *Phi, float mu, const float *y, int B, const cs_step_options *o,
+                              int32_t *support, float *z, float *resid, bool gram_ready, cudaStream_t st) {
+    const int T = o->T < 0 ? plan->cfg.T : o->T;
+    if (o->solver == CS_SOLVER_NIHT) return launch_niht(plan, Phi, mu, y, B, T, support, z, resid, st);
+    if (o->solver == CS_SOLVER_OMP) return launch_omp(plan, Phi, y, B, support, z, resid, st);
+    return launch_recover(plan, Phi, mu, y, B, support, z, resid, gram_ready, st, T,
+                          o->warm_start ? o->support_prev : nullptr, o->warm_start ? o->z_prev : nullptr, o->gamma,
+                          o->gamma > 0.f ? o->support_prev : nullptr, o->gamma > 0.f ? o->z_prev : nullptr);
+}
+
+cs_status cs_recover_ex(cs_plan *plan, const float *Phi, float mu, const float *y, int32_t B,
+                        const cs_step_options *opt, int32_t *support, float *z, float *resid, void *stream) {
+    if (opt == nullptr) return cs_recover(plan, Phi, mu, y, B, support, z, resid, stream);
+    if (plan == nullptr || Phi == nullptr || y == nullptr || support == nullptr) return CS_ERR_NULL;
+    if (B <= 0 || B > plan->cfg.max_tokens) return CS_ERR_SHAPE;
+    if (!isfinite(mu) || !(mu > 0.f)) return CS_ERR_NONFINITE;
+    cs_status s = check_options(plan, opt, false);
+    if (s != CS_OK) return s;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (opt->support_prev != nullptr) {
+        s = launch_check_support(plan, opt->support_prev, B, st);
+        if (s != CS_OK) return s;
+    }
+    s = recover_with(plan, Phi, mu, y, B, opt, support, z, resid, false, st);
+    if (s != CS_OK) return s;
+    if (opt->delta_out != nullptr || opt->drift_out != nullptr)
+        s = launch_support_drift(plan, opt->support_prev, support, B, opt->delta_out, opt->drift_out, st);
+    return s;
+}
+
+cs_status cs_sketch_srht(cs_plan *plan, const uint32_t *sign_bits, const int32_t *rows, const float *h, int32_t B,
+                         float *y, void *stream) {
+    if (plan == nullptr || sign_bits == nullptr || rows == nullptr || h == nullptr || y == nullptr) return CS_ERR_NULL;
+    if (B <= 0 || B > plan->cfg.max_tokens) return CS_ERR_SHAPE;
+    return launch_sketch_srht(plan, sign_bits, rows, h, B, y, static_cast<cudaStream_t>(stream));
 }
 
 cs_status cs_uds_budget(cs_plan *plan, const float *logits, int32_t B, int32_t V, float m_base, float gamma,
@@ -333,6 +403,92 @@ cs_status cs_layer_step(cs_plan *plan, const cs_layer *layer, const float *x, in
     if (s != CS_OK) return s;
     // supports produced by the recovery are valid by construction: no device check here
     return exec_dispatch(plan, layer, n, sup, B, layer->add_residual ? x : nullptr, x_out, false, st);
+}
+
+cs_status cs_layer_step_ex(cs_plan *plan, const cs_layer *layer, const float *x, int32_t B,
+                           const cs_step_options *opt, float *x_out, int32_t *support_out, float *z_out,
+                           float *resid_out, void *stream) {
+    if (opt == nullptr) return cs_layer_step(plan, layer, x, B, x_out, support_out, z_out, resid_out, stream);
+    if (plan == nullptr || x == nullptr || x_out == nullptr) return CS_ERR_NULL;
+    cs_status s = check_weights(layer);
+    if (s != CS_OK) return s;
+    const bool srht = opt->srht_sign != nullptr;
+    if (layer->Phi == nullptr || (!srht && layer->S == nullptr)) return CS_ERR_NULL;
+    if (B <= 0 || B > plan->cfg.max_tokens) return CS_ERR_SHAPE;
+    if (!isfinite(layer->mu) || !(layer->mu > 0.f)) return CS_ERR_NONFINITE;
+    if (!aligned16(x) || !aligned16(x_out) || (!srht && !aligned16(layer->S)) ||
+        (layer->rms_gamma != nullptr && !aligned16(layer->rms_gamma)))
+        return CS_ERR_UNSUPPORTED;
+    s = check_options(plan, opt, true);
+    if (s != CS_OK) return s;
+    const bool norm = layer->rms_gamma != nullptr;
+    if (srht && norm) return CS_ERR_UNSUPPORTED;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (opt->support_prev != nullptr) {
+        s = launch_check_support(plan, opt->support_prev, B, st);
+        if (s != CS_OK) return s;
+    }
+    const float *n = norm ? plan->n_buf : x;
+    const float *residual = layer->add_residual ? x : nullptr;
+    if (opt->reuse_support) {   // no estimation this step: the previous supports execute
+        if (norm) {   // the sketch kernel also forms the normalised input
+            s = launch_sketch(plan, layer->S, x, layer->rms_gamma, B, plan->y_buf, plan->n_buf, nullptr, 0.f, st);
+            if (s != CS_OK) return s;
+        }
+        if (support_out != nullptr)
+            CS_CUDA_TRY(plan, cudaMemcpyAsync(support_out, opt->support_prev, (size_t)B * plan->cfg.k * sizeof(int32_t),
+                                              cudaMemcpyDeviceToDevice, st));
+        return exec_dispatch(plan, layer, n, opt->support_prev, B, residual, x_out, false, st);
+    }
+    if (srht) s = launch_sketch_srht(plan, opt->srht_sign, opt->srht_rows, x, B, plan->y_buf, st);
+    else s = launch_sketch(plan, layer->S, x, layer->rms_gamma, B, plan->y_buf, norm ? plan->n_buf : nullptr, layer->Phi,
+                           layer->mu, st);
+    if (s != CS_OK) return s;
+    int32_t *sup = support_out != nullptr ? support_out : plan->sup_buf;
+    s = recover_with(plan, layer->Phi, layer->mu, plan->y_buf, B, opt, sup, z_out, resid_out, !srht, st);
+    if (s != CS_OK) return s;
+    if (opt->delta_out != nullptr || opt->drift_out != nullptr) {
+        s = launch_support_drift(plan, opt->support_prev, sup, B, opt->delta_out, opt->drift_out, st);
+        if (s != CS_OK) return s;
+    }
+    return exec_dispatch(plan, layer, n, sup, B, residual, x_out, false, st);
+}
+
+cs_status cs_layer_step_fallback(cs_plan *plan, cs_plan *dense, const cs_layer *layer, const float *x, int32_t B,
+                                 const cs_step_options *opt, float tau, float *x_out, int32_t *support_out,
+                                 float *z_out, float *resid_out, int32_t *flags_out, int32_t *n_fallback,
+                                 void *stream) {
+    if (plan == nullptr || dense == nullptr || n_fallback == nullptr) return CS_ERR_NULL;
+    const cs_config &a = plan->cfg, &b = dense->cfg;
+    if (a.d != b.d || a.d_ff != b.d_ff || a.group != b.group || a.m != b.m || a.w_dtype != b.w_dtype || b.k < a.k ||
+        B > b.max_tokens)
+        return CS_ERR_SHAPE;
+    if (!isfinite(tau) || tau < 0.f) return CS_ERR_NONFINITE;
+    if (opt != nullptr && opt->reuse_support) return CS_ERR_UNSUPPORTED;
+    if (x_out == x) return CS_ERR_UNSUPPORTED;   // the second pass reads x again
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    float *resid = resid_out != nullptr ? resid_out : plan->resid_buf;
+    cs_status s = cs_layer_step_ex(plan, layer, x, B, opt, x_out, support_out, z_out, resid, stream);
+    if (s != CS_OK) return s;
+    s = launch_confidence(plan, plan->y_buf, resid, B, tau, flags_out != nullptr ? flags_out : plan->fb_flags, plan->fb_list,
+                          plan->fb_count, st);
+    if (s != CS_OK) return s;
+    int32_t n_low = 0;
+    CS_CUDA_TRY(plan, cudaMemcpyAsync(&n_low, plan->fb_count, sizeof n_low, cudaMemcpyDeviceToHost, st));
+    CS_CUDA_TRY(plan, cudaStreamSynchronize(st));
+    *n_fallback = n_low;
+    if (n_low == 0) return CS_OK;
+    // the untrusted tokens alone, through the denser plan, and back into their rows
+    s = launch_gather_rows(plan, x, plan->fb_list, n_low, dense->x_host_in, st);
+    if (s != CS_OK) return s;
+    cs_step_options second;
+    memset(&second, 0, sizeof second);
+    second.T = -1;
+    if (opt != nullptr) { second.solver = opt->solver; second.srht_sign = opt->srht_sign; second.srht_rows = opt->srht_rows; }
+    if (second.solver == CS_SOLVER_OMP && b.k > 64) second.solver = CS_SOLVER_IHT;
+    s = cs_layer_step_ex(dense, layer, dense->x_host_in, n_low, &second, dense->x_host_out, nullptr, nullptr, nullptr, stream);
+    if (s != CS_OK) return s;
+    return launch_scatter_rows(plan, dense->x_host_out, plan->fb_list, n_low, x_out, st);
 }
 
 cs_status cs_layer_step_host(cs_plan *plan, const cs_layer *layer, const float *x_host, int32_t B,

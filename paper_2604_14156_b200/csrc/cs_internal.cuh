@@ -39,6 +39,10 @@ struct cs_plan {
     int32_t *sup_buf;  // [max_tokens, k]
     float *partial;    // [kGatherMaxTokens, nx_max, d] partial down-projections of the gather path
     float *gram;       // [G, pitch] I - mu Phi^T Phi of the layer being recovered, pitch = 32 ceil(G/32)
+    float *resid_buf;     // [max_tokens] residual norms when the caller wants none (confidence fallback)
+    int32_t *fb_flags;    // [max_tokens] confidence fallback: 1 = the token's recovery is not trusted
+    int32_t *fb_list;     // [max_tokens] those tokens, ascending
+    int32_t *fb_count;    // [1] their number
     int32_t *slot_table;  // [max_tokens, kSlotTablePitch] small-batch step: slot -> group of the recovery in flight
     unsigned *ticket;     // [max_tokens] arrival counters of the sketch CTAs (zero between launches)
     float *hbar;       // [d] mean prompt hidden state
@@ -110,7 +114,18 @@ cs_status launch_sketch(cs_plan *plan, const float *S, const float *x, const flo
 // gram_ready: plan->gram already holds this Phi's matrix (the sketch launch before formed it).
 cs_status launch_recover(cs_plan *plan, const float *Phi, float mu, const float *y, int B,
                          int32_t *support, float *z, float *resid, bool gram_ready, cudaStream_t st,
-                         int T = -1 /* the plan's */, const int32_t *sup0 = nullptr, const float *z0 = nullptr);
+                         int T = -1 /* the plan's */, const int32_t *sup0 = nullptr, const float *z0 = nullptr,
+                         float gamma = 0.f /* temporal term */, const int32_t *sup_prev = nullptr,
+                         const float *z_prev = nullptr);
+// the other estimators (solvers.cu)
+cs_status prepare_solvers(cs_plan *plan);
+cs_status launch_niht(cs_plan *plan, const float *Phi, float mu_fallback, const float *y, int B, int T,
+                      int32_t *support, float *z, float *resid, cudaStream_t st);
+cs_status launch_omp(cs_plan *plan, const float *Phi, const float *y, int B, int32_t *support, float *z, float *resid,
+                     cudaStream_t st);
+// the structured sketch (srht.cu)
+cs_status launch_sketch_srht(cs_plan *plan, const uint32_t *sign_bits, const int32_t *rows, const float *h, int B, float *y,
+                             cudaStream_t st);
 // check: validate the supports on the device (ascending, distinct, in range) inside the same launch
 cs_status launch_ffn_gather(cs_plan *plan, const cs_layer *layer, const float *h, const int32_t *support,
                             int B, const float *residual, float *out, bool check, cudaStream_t st);
@@ -125,7 +140,12 @@ cs_status launch_ffn_gather_spec(cs_plan *plan, const cs_layer *layer, const flo
                                  float *out, cudaStream_t st);
 cs_status prepare_ffn_gather(cs_plan *plan);
 cs_status launch_support_drift(cs_plan *plan, const int32_t *prev, const int32_t *cur, int B, int32_t *drift,
-                               cudaStream_t st);
+                               float *ratio, cudaStream_t st);
+// confidence fallback (control.cu): flags tokens whose relative residual exceeds tau, lists them, moves rows
+cs_status launch_confidence(cs_plan *plan, const float *y, const float *resid, int B, float tau, int32_t *flags,
+                            int32_t *list, int32_t *count, cudaStream_t st);
+cs_status launch_gather_rows(cs_plan *plan, const float *src, const int32_t *list, int n, float *dst, cudaStream_t st);
+cs_status launch_scatter_rows(cs_plan *plan, const float *src, const int32_t *list, int n, float *dst, cudaStream_t st);
 cs_status launch_uds_budget(cs_plan *plan, const float *logits, int B, int V, float m_base, float gamma,
                             int m_min, int m_max, float *H, int32_t *m_t, cudaStream_t st);
 cs_status launch_check_support(cs_plan *plan, const int32_t *support, int B, cudaStream_t st);

@@ -17,7 +17,7 @@ __global__ void __launch_bounds__(32 * NW)
 recover_kernel(const float *__restrict__ Phi, const float *__restrict__ gram, float mu, const float *__restrict__ y,
                int m, int G, int k, int T, int32_t *__restrict__ support, float *__restrict__ z_out,
                float *__restrict__ resid_out, const int32_t *__restrict__ sup0, const float *__restrict__ z0,
-               DeviceStatus *status) {
+               float tgamma, const int32_t *__restrict__ sup_prev, const float *__restrict__ z_prev, DeviceStatus *status) {
     __shared__ RecoverSmem<NW, KC> s;
     const int g = threadIdx.x, t = blockIdx.x;
     pdl_launch_dependents();
@@ -30,11 +30,12 @@ recover_kernel(const float *__restrict__ Phi, const float *__restrict__ gram, fl
                              z_out != nullptr ? z_out + (size_t)t * k : nullptr,
                              resid_out != nullptr ? resid_out + t : nullptr,
                              sup0 != nullptr ? sup0 + (size_t)t * k : nullptr, z0 != nullptr ? z0 + (size_t)t * k : nullptr,
-                             status, phc, [] {}, [](int, int) {}, [] {});
+                             tgamma, sup_prev != nullptr ? sup_prev + (size_t)t * k : nullptr,
+                             z_prev != nullptr ? z_prev + (size_t)t * k : nullptr, status, phc, [] {}, [](int, int) {}, [] {});
 }
 
 typedef void (*RecoverFn)(const float *, const float *, float, const float *, int, int, int, int, int32_t *, float *, float *,
-                          const int32_t *, const float *, DeviceStatus *);
+                          const int32_t *, const float *, float, const int32_t *, const float *, DeviceStatus *);
 static int recover_kc(int k) { return k <= 56 ? (k + 7) / 8 : 0; }
 template <int NW> static RecoverFn recover_fn_kc(int k) {
     switch (recover_kc(k)) {
@@ -58,7 +59,7 @@ static RecoverFn recover_fn(int G, int k) {
 }
 cs_status launch_recover(cs_plan *plan, const float *Phi, float mu, const float *y, int B, int32_t *support,
                          float *z, float *resid, bool gram_ready, cudaStream_t st, int T, const int32_t *sup0,
-                         const float *z0) {
+                         const float *z0, float gamma, const int32_t *sup_prev, const float *z_prev) {
     const cs_config &c = plan->cfg;
     const int G = plan->G;
     StageTimer timer(plan, CS_STAGE_RECOVER, st);
@@ -68,7 +69,8 @@ cs_status launch_recover(cs_plan *plan, const float *Phi, float mu, const float 
         CS_CUDA_TRY(plan, cudaGetLastError());
     }
     launch_pdl(pdl_for(plan, B), recover_fn(G, c.k), dim3(B), dim3(gram_pitch(G)), 0, st, Phi,
-               (const float *)plan->gram, mu, y, c.m, G, c.k, T < 0 ? c.T : T, support, z, resid, sup0, z0, plan->status);
+               (const float *)plan->gram, mu, y, c.m, G, c.k, T < 0 ? c.T : T, support, z, resid, sup0, z0, 2.f * mu * gamma, sup_prev,
+               z_prev, plan->status);
     plan->launches++;
     CS_CUDA_TRY(plan, cudaGetLastError());
     return CS_OK;
@@ -80,7 +82,7 @@ cs_status launch_recover(cs_plan *plan, const float *Phi, float mu, const float 
 constexpr int kDriftThreads = kMaxG;
 __global__ void __launch_bounds__(kDriftThreads)
 support_drift_kernel(const int32_t *__restrict__ prev, const int32_t *__restrict__ cur, int k,
-                     int32_t *__restrict__ drift) {
+                     int32_t *__restrict__ drift, float *__restrict__ ratio) {
     const int t = blockIdx.x, j = threadIdx.x;
     const int32_t *p = prev + (size_t)t * k;
     int missing = 0;
@@ -94,12 +96,16 @@ support_drift_kernel(const int32_t *__restrict__ prev, const int32_t *__restrict
         missing = !(lo < k && p[lo] == e);
     }
     const int n = __syncthreads_count(missing);
-    if (j == 0) drift[t] = 2 * n;
+    if (j == 0) {
+        if (drift != nullptr) drift[t] = 2 * n;
+        // D_t = |S_t sym.diff S_{t-1}| / |S_t union S_{t-1}| (Sec. 15): both rows have k entries, so the union has k + n
+        if (ratio != nullptr) ratio[t] = (float)(2 * n) / (float)(k + n);
+    }
 }
 
 cs_status launch_support_drift(cs_plan *plan, const int32_t *prev, const int32_t *cur, int B, int32_t *drift,
-                               cudaStream_t st) {
-    support_drift_kernel<<<B, kDriftThreads, 0, st>>>(prev, cur, plan->cfg.k, drift);
+                               float *ratio, cudaStream_t st) {
+    support_drift_kernel<<<B, kDriftThreads, 0, st>>>(prev, cur, plan->cfg.k, drift, ratio);
     plan->launches++;
     CS_CUDA_TRY(plan, cudaGetLastError());
     return CS_OK;

@@ -175,7 +175,8 @@ __device__ __forceinline__ void recover_token(RecoverSmem<NW, KC> &s, const int 
                                               const MSource M, float mu, const float *__restrict__ y, int m, int G, int k, int T, int32_t *__restrict__ support,
                                               float *__restrict__ z_out, float *__restrict__ resid_out,
                                               const int32_t *__restrict__ sup0, const float *__restrict__ z0,
-                                              DeviceStatus *status, const float (&phc)[32], TableReady table_ready,
+                                              const float tgamma, const int32_t *__restrict__ sup_prev,
+                                              const float *__restrict__ z_prev, DeviceStatus *status, const float (&phc)[32], TableReady table_ready,
                                               SlotChanged slot_changed, TableFinal table_final) {
     constexpr int GP = 32 * NW;
     constexpr int NV = RecoverSmem<NW, KC>::NV;
@@ -220,6 +221,16 @@ __device__ __forceinline__ void recover_token(RecoverSmem<NW, KC> &s, const int 
     bool kept = warm ? s.slot[g] >= 0 : g < k;
     int slot = warm ? max(s.slot[g], 0) : g;
     float v = 0.f;
+    // Temporal regulariser (Sec. 5), tgamma = 2 mu gamma: the step gains  tgamma (z_prev - z)_g.  z_prev is the
+    // k-sparse estimate of the previous decoding step (sup_prev ascending, z_prev its values).
+    float zprev_g = 0.f;
+    if (tgamma != 0.f && sup_prev != nullptr) {
+        for (int j = 0; j < k; ++j)
+            if (ld_dep(sup_prev + j) == g) zprev_g = ld_dep(z_prev + j);
+        if (warm && kept) {   // v holds this entry's value in the current iterate
+            if constexpr (KC > 0) v = s.val[0][slot]; else v = s.val[0][g];
+        }
+    }
     if constexpr (KC > 0) {
         if (warm) {   // the entries that go with the warm list
 #pragma unroll
@@ -265,7 +276,9 @@ __device__ __forceinline__ void recover_token(RecoverSmem<NW, KC> &s, const int 
                 a0 = fmaf(mreg[4 * j], zq.x, a0); a1 = fmaf(mreg[4 * j + 1], zq.y, a1);
                 a2 = fmaf(mreg[4 * j + 2], zq.z, a2); a3 = fmaf(mreg[4 * j + 3], zq.w, a3);
             }
+            const float zcur = kept ? v : 0.f;   // this entry of the current iterate (v: its value from the step before)
             v = (a0 + a1) + (a2 + a3);
+            if (tgamma != 0.f) v = fmaf(tgamma, zprev_g - zcur, v);
         }
         // Keys are |v| (entries past G get -2: they precede nothing).  A NaN has no place in the order:
         // it is ranked as a zero, so that the fast test below (integer order) and the exact ranks

@@ -180,7 +180,7 @@ sketch_kernel(const float *__restrict__ S, const float *__restrict__ x, const fl
         recover_token<kSketchRecNW, kSketchRecKC, 1>(
             rs, g, Phi, src, mu, y + (size_t)t * m, m, G, k, ra.T,
             ra.support != nullptr ? ra.support + (size_t)t * k : nullptr, ra.z != nullptr ? ra.z + (size_t)t * k : nullptr,
-            ra.resid != nullptr ? ra.resid + t : nullptr, nullptr, nullptr, ra.status, phc,
+            ra.resid != nullptr ? ra.resid + t : nullptr, nullptr, nullptr, 0.f, nullptr, nullptr, ra.status, phc,
             [&] {   // the first iterate's table goes out, then the launch's trigger
                 if (g < k) st_visible(table + g, rs.idx[g]);
                 __threadfence();
