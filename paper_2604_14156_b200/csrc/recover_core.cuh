@@ -387,6 +387,7 @@ __device__ __forceinline__ void recover_token(RecoverSmem<NW, KC> &s, const int 
             float ss = 0.f;
             for (int row = g; row < m; row += GP) {
                 float a = 0.f;
+#pragma unroll 8
                 for (int j = 0; j < k; ++j) a = fmaf(M.phi(Phi, row, s.idx[j], G), s.val[T & 1][j], a);
                 const float r = s.y[row] - a;
                 ss = fmaf(r, r, ss);
