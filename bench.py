@@ -45,7 +45,9 @@ UNIT = "tokens/s"
 # ncu captures summarised under profiles/, keyed by (workload, k).  An entry is removed when its
 # kernel changes and comes back with the next capture; a missing entry reports null.
 NCU_TRAFFIC = {
-    ("l2_7b_b1", 22): 69.24e6 + 1.60e6,                       # ffn_gather_kernel
+    ("l2_7b_b1", 22): 69.24e6 + 1.34e6,                       # ffn_gather_kernel
+    ("l2_7b_b64", 22): 181.47e6 + 4.24e6 + 95.85e6 + 3.71e6,  # ffn_gateup_swap_kernel + ffn_down_swap_kernel
+    ("l2_13b_prompt", 27): 207.11e6 + 10.73e6 + 58.03e6 + 4.08e6,  # ffn_gateup_mma_kernel + ffn_down_wide_kernel
 }
 GRAPH_STEPS = 64          # most steps captured per CUDA graph
 N_TOKEN_BATCHES = 16      # distinct input batches rotated through
