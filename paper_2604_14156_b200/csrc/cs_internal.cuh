@@ -64,6 +64,7 @@ struct cs_plan {
     int mma_min_tokens;  // smallest decode batch that takes it
     int mma_slices;      // most list slices the down GEMM is split into
     int last_slices;
+    int pair_key_ng, pair_key_mtiles, pair_count;   // prompt gate/up: paired-tile count of the last shape seen
     float *x_host_in;  // [max_tokens, d] staging for the host-buffer entry point
     float *x_host_out; // [max_tokens, d]
     cudaEvent_t ev[2 * CS_STAGE_COUNT];  // start/stop per stage

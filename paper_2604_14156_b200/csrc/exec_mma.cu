@@ -27,6 +27,9 @@
 // CTA drains and exits.
 #include <cuda.h>
 
+#include <algorithm>
+#include <vector>
+
 #include "cs_internal.cuh"
 
 namespace cs {
@@ -317,6 +320,108 @@ ffn_gateup_mma_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_con
     epilogue_done(t, warp);
 }
 
+// ---- gate / up for one shared support (the prompt-level variant): single and paired token tiles ---------
+// A 128 x 256 tile with both operands streamed per 64-wide k block takes in 0.0117 bytes per flop, which at
+// the rate of the tensor pipe is more than the SMs can take in from L2 (the kernel above sits at 13.5 TB/s
+// of ingest with the pipe 63 % busy).  A CTA that owns TWO token tiles of one group shares every weight
+// tile between them: 64 KB per stage for twice the flops, two accumulators in the 512 tensor-memory
+// columns.  Paired tiles alone would waste the last wave (a pair is twice the work), so one launch mixes
+// them: CTAs [0, n_pair) take pair slots, the CTAs behind them split the remaining pair slots into single
+// tiles; the hardware hands CTAs out in index order, so the singles fill the SMs as the pairs finish.
+// Pair slot q = (group q % ng, token tiles 2 (q / ng) and 2 (q / ng) + 1).
+__global__ void __launch_bounds__(kMmaThreads, 1)
+ffn_gateup_tiles_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_g,
+                        const __grid_constant__ CUtensorMap tm_u, const int32_t *__restrict__ glist, int ng, int n_pair,
+                        int mtiles, int M, int d, int act_ld, __nv_bfloat16 *__restrict__ act, DeviceStatus *status) {
+    extern __shared__ uint8_t smem_raw[];
+    const int c = blockIdx.x;
+    const bool pair = c < n_pair;
+    const int q = pair ? c : n_pair + ((c - n_pair) >> 1);
+    const int gi = q % ng, mt0 = 2 * (q / ng) + (pair ? 0 : ((c - n_pair) & 1));
+    if (mt0 >= mtiles) return;                                   // the odd half of a last, incomplete pair slot
+    const int ntile = (pair && mt0 + 1 < mtiles) ? 2 : 1;
+    const int g = glist[gi];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    uint8_t *base = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    Barriers *bars = reinterpret_cast<Barriers *>(base + kRingBytesMma);
+    const int stage_bytes = ntile * kABytes + kBBytes;           // 48 KB or 64 KB
+    const int stages = kRingBytesMma / stage_bytes;              // 4 or 3
+    const uint32_t tcols = ntile == 2 ? 512u : 256u;
+    setup_cta(bars, warp, tcols);
+    const int kblocks = d / BK;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            int s = 0, ph = 1;                                   // ring slot and the parity of its previous use
+            for (int kb = 0; kb < kblocks; ++kb, ++s) {
+                if (s == stages) { s = 0; ph ^= 1; }
+                if (kb >= stages && !mbar_wait(&bars->empty[s], ph, bars, status)) break;
+                uint8_t *st = base + (size_t)s * stage_bytes;
+                mbar_expect_tx(&bars->full[s], stage_bytes);
+                tma_load_2d(st, &tm_x, kb * BK, mt0 * BM, &bars->full[s]);
+                if (ntile == 2) tma_load_2d(st + kABytes, &tm_x, kb * BK, (mt0 + 1) * BM, &bars->full[s]);
+                uint8_t *b = st + ntile * kABytes;
+                tma_load_2d(b, &tm_g, kb * BK, g * 128, &bars->full[s]);
+                tma_load_2d(b + kBBytes / 2, &tm_u, kb * BK, g * 128, &bars->full[s]);
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            constexpr uint32_t idesc = make_idesc(false);
+            const uint32_t tmem = bars->tmem_base;
+            bool ok = true;
+            int s = 0, ph = 0;
+            for (int kb = 0; kb < kblocks && ok; ++kb, ++s) {
+                if (s == stages) { s = 0; ph ^= 1; }
+                ok = mbar_wait(&bars->full[s], ph, bars, status);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t a0 = smem_u32(base + (size_t)s * stage_bytes), b0 = a0 + ntile * kABytes;
+#pragma unroll
+                for (int k4 = 0; k4 < BK / 16; ++k4) {
+                    const uint64_t bd = desc_sw128(b0 + k4 * 32, 16);
+                    tc_mma(tmem, desc_sw128(a0 + k4 * 32, 16), bd, idesc, (kb | k4) != 0);
+                    if (ntile == 2) tc_mma(tmem + 256, desc_sw128(a0 + kABytes + k4 * 32, 16), bd, idesc, (kb | k4) != 0);
+                }
+                tc_commit(&bars->empty[s]);
+            }
+            if (ok) tc_commit(&bars->acc_ready);
+        }
+    } else {
+        const int qd = warp & 3;                   // TMEM lane quarter this warp may read
+        const int row = qd * 32 + lane;
+        if (mbar_wait(&bars->acc_ready, 0, bars, status)) {
+            tc_fence_after();
+            for (int tt = 0; tt < ntile; ++tt) {
+                const int m = (mt0 + tt) * BM + row;
+                const uint32_t tbase = bars->tmem_base + ((uint32_t)(qd * 32) << 16) + (uint32_t)(tt * 256);
+#pragma unroll 1
+                for (int cc = 0; cc < 4; ++cc) {
+                    uint32_t gv[32], uv[32];
+                    tc_ld32(tbase + cc * 32, gv);
+                    tc_ld32(tbase + 128 + cc * 32, uv);
+                    tc_wait_ld();
+                    uint32_t packed[16];
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) {
+                        const float a0 = silu_f(__uint_as_float(gv[2 * j])) * __uint_as_float(uv[2 * j]);
+                        const float a1 = silu_f(__uint_as_float(gv[2 * j + 1])) * __uint_as_float(uv[2 * j + 1]);
+                        const __nv_bfloat162 p = __floats2bfloat162_rn(a0, a1);
+                        packed[j] = *reinterpret_cast<const uint32_t *>(&p);
+                    }
+                    if (m < M) {
+                        uint4 *dst = reinterpret_cast<uint4 *>(act + (size_t)m * act_ld + (size_t)gi * 128 + cc * 32);
+#pragma unroll
+                        for (int j = 0; j < 4; ++j)
+                            dst[j] = make_uint4(packed[4 * j], packed[4 * j + 1], packed[4 * j + 2], packed[4 * j + 3]);
+                    }
+                }
+            }
+        }
+    }
+    teardown_cta(bars, warp, tcols);
+}
+
 // ---- down -------------------------------------------------------------------------------------
 // grid (d / 256, token tiles, slices).  Slice z covers list entries [z*ng/Z, (z+1)*ng/Z).
 template <bool SPLIT>
@@ -582,9 +687,10 @@ ffn_gateup_swap_kernel(const __grid_constant__ CUtensorMap tm_g, const __grid_co
             const uint32_t idesc = make_idesc_rt(NB, false, false);
             const uint32_t tmem = bars->tmem_base;
             bool ok = true;
-            for (int kb = 0; kb < kblocks && ok; ++kb) {
-                const int s = kb % stages;
-                ok = mbar_wait(&bars->full[s], (kb / stages) & 1, bars, status);
+            int s = 0, ph = 0;
+            for (int kb = 0; kb < kblocks && ok; ++kb, ++s) {
+                if (s == stages) { s = 0; ph ^= 1; }
+                ok = mbar_wait(&bars->full[s], ph, bars, status);
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t a_g = smem_u32(base + (size_t)s * stage_bytes), a_u = a_g + kABytes;
@@ -720,9 +826,10 @@ ffn_down_swap_kernel(const __grid_constant__ CUtensorMap tm_wd, const __grid_con
             const uint32_t idesc = make_idesc_rt(NB, true, true);
             const uint32_t tmem = bars->tmem_base;
             bool ok = true;
-            for (int kb = 0; kb < kblocks && ok; ++kb) {
-                const int s = kb % stages;
-                ok = mbar_wait(&bars->full[s], (kb / stages) & 1, bars, status);
+            int s = 0, ph = 0;
+            for (int kb = 0; kb < kblocks && ok; ++kb, ++s) {
+                if (s == stages) { s = 0; ph ^= 1; }
+                ok = mbar_wait(&bars->full[s], ph, bars, status);
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t a0 = smem_u32(base + (size_t)s * stage_bytes), b0 = a0 + CPC * kABytes;
@@ -1000,7 +1107,38 @@ bool make_map(CUtensorMap *map, const void *base, uint64_t inner, uint64_t outer
 
 }  // namespace
 
+// How many of the pair slots a mixed launch runs as paired tiles: CTAs are handed out in index order to
+// whichever SM is free first, pairs first.  Measured on B200, a pair takes about 1.8 single-tile times
+// (both kinds are bound by what shared memory can serve: the tensor pipe reads 12 KB of operands per
+// 128 x 256 x 16 instruction while TMA refills the ring, and a pair saves only the second refill of
+// the weight tile), so pairs pay off where they fix the last wave: 176 tiles on 148 SMs (two waves
+// of singles, one of pairs), 864 tiles (six waves against three), not 432 (three full waves).
+// The count with the shortest predicted makespan wins if it beats all-singles by 8 % or more.
+constexpr double kPairCost = 1.8;
+static int best_pair_count(int slots, int mtiles, int ng, int sms) {
+    int best = 0;
+    double best_t = 1e30;
+    std::vector<double> free_at(sms);
+    for (int n_pair = 0; n_pair <= slots; ++n_pair) {
+        std::fill(free_at.begin(), free_at.end(), 0.0);
+        auto run = [&](double cost) {
+            auto it = std::min_element(free_at.begin(), free_at.end());
+            *it += cost;
+        };
+        for (int q = 0; q < n_pair; ++q) run(2 * (q / ng) + 1 < mtiles ? kPairCost : 1.0);
+        for (int q = n_pair; q < slots; ++q) {
+            run(1.0);
+            if (2 * (q / ng) + 1 < mtiles) run(1.0);
+        }
+        const double t = *std::max_element(free_at.begin(), free_at.end());
+        if (n_pair == 0) { best_t = t * 0.92; continue; }   // what pairs have to beat
+        if (t <= best_t + 1e-9) { best_t = t; best = n_pair; }
+    }
+    return best;
+}
+
 cs_status prepare_ffn_mma(cs_plan *plan) {
+    CS_CUDA_TRY(plan, cudaFuncSetAttribute(ffn_gateup_tiles_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMmaSmem));
     CS_CUDA_TRY(plan, cudaFuncSetAttribute(ffn_down_wide_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMmaSmem));
     CS_CUDA_TRY(plan, cudaFuncSetAttribute(ffn_gateup_mma_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMmaSmem));
     CS_CUDA_TRY(plan, cudaFuncSetAttribute(ffn_gateup_mma_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMmaSmem));
@@ -1042,12 +1180,27 @@ cs_status launch_ffn_mma(cs_plan *plan, const cs_layer *L, const void *X, const 
         !make_map(&tm_act_lo, split ? act_lo : act, act_ld, M, act_ld, BM) ||
         !make_map(&tm_wd, L->Wd_t, c.d, c.d_ff, c.d, BK))
         return record_cuda(plan, cudaErrorInvalidValue, "cuTensorMapEncodeTiled");
+    // One shared support whose size the host knows: how many pair slots run as paired token tiles (the
+    // schedule of this shape, computed once); none leaves the launch to the single-tile kernel.
+    int n_pair = 0;
+    const int slots = ng_host * ((mtiles + 1) / 2);
+    if (!split && ng_dev == nullptr && mask == nullptr && ng_host > 0) {
+        if (plan->pair_key_ng != ng_host || plan->pair_key_mtiles != mtiles) {
+            plan->pair_count = best_pair_count(slots, mtiles, ng_host, plan->sm_count);
+            plan->pair_key_ng = ng_host; plan->pair_key_mtiles = mtiles;
+        }
+        n_pair = plan->pair_count;
+    }
     {
         StageTimer timer(plan, CS_STAGE_EXEC, st);
         if (split)
             ffn_gateup_mma_kernel<true><<<dim3(grid_g, mtiles), kMmaThreads, kMmaSmem, st>>>(
                 tm_x, tm_x_lo, tm_g, tm_u, glist, ng_dev, ng_host, M, c.d, act_ld, mask, act, act_lo, plan->status);
-        else
+        else if (n_pair > 0) {
+            // one shared support, its size known on the host: paired and single token tiles in one launch
+            ffn_gateup_tiles_kernel<<<dim3(n_pair + 2 * (slots - n_pair)), kMmaThreads, kMmaSmem, st>>>(
+                tm_x, tm_g, tm_u, glist, ng_host, n_pair, mtiles, M, c.d, act_ld, act, plan->status);
+        } else
             ffn_gateup_mma_kernel<false><<<dim3(grid_g, mtiles), kMmaThreads, kMmaSmem, st>>>(
                 tm_x, tm_x_lo, tm_g, tm_u, glist, ng_dev, ng_host, M, c.d, act_ld, mask, act, act_lo, plan->status);
         plan->launches++;
