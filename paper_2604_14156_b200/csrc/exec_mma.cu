@@ -42,7 +42,10 @@ constexpr int kABytes = BM * BK * 2;   // 16 KB
 constexpr int kBBytes = BN * BK * 2;   // 32 KB
 constexpr int kRingBytesMma = 4 * (kABytes + kBBytes);   // 192 KB of operand tiles
 constexpr int kMmaThreads = 192;
-constexpr int kSwapMaxThreads = 64 + 4 * 128;   // decode kernels: up to four epilogue slices of four warps
+// Epilogue warps come in slices of four (a warp may read the tensor-memory lane quarter warp % 4); a kernel
+// launched with 64 + 128 S threads drains its accumulators with S slices, each taking every S-th chunk.
+constexpr int kSwapMaxThreads = 64 + 4 * 128;
+constexpr int kTileThreads = kSwapMaxThreads;   // the 128-token-tile kernels: four slices
 constexpr uint32_t kSpinLimit = 1u << 20;
 constexpr size_t kMmaSmem = 1024 + (size_t)kRingBytesMma + 256;
 
@@ -245,7 +248,7 @@ __device__ __forceinline__ float silu_f(float x) { return x / (1.f + __expf(-x))
 
 // ---- gate / up --------------------------------------------------------------------------------
 template <bool SPLIT>
-__global__ void __launch_bounds__(kMmaThreads, 1)
+__global__ void __launch_bounds__(kTileThreads, 1)
 ffn_gateup_mma_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_x_lo,
                       const __grid_constant__ CUtensorMap tm_g, const __grid_constant__ CUtensorMap tm_u,
                       const int32_t *__restrict__ glist, const int32_t *__restrict__ ng_dev, int ng_host, int M,
@@ -278,6 +281,7 @@ ffn_gateup_mma_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_con
         if (lane == 0) mma_loop<false, SPLIT>(t, kblocks, status);
     } else {
         const int q = warp & 3;                    // TMEM lane quarter this warp may read
+        const int slice = (warp - 2) >> 2, nslice = ((int)(blockDim.x >> 5) - 2) >> 2;
         const int row = q * 32 + lane, m = mt * BM + row;
         if (mbar_wait(&t.bars->acc_ready, 0, t.bars, status)) {
             tc_fence_after();
@@ -285,7 +289,7 @@ ffn_gateup_mma_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_con
             float keep = 1.f;
             if (mask != nullptr && m < M) keep = ((mask[(size_t)m * 4 + (g >> 5)] >> (g & 31)) & 1u) ? 1.f : 0.f;
 #pragma unroll 1
-            for (int c = 0; c < 4; ++c) {
+            for (int c = slice; c < 4; c += nslice) {
                 uint32_t gv[32], uv[32];
                 tc_ld32(tbase + c * 32, gv);
                 tc_ld32(tbase + 128 + c * 32, uv);
@@ -330,7 +334,7 @@ ffn_gateup_mma_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_con
 // them: CTAs [0, n_pair) take pair slots, the CTAs behind them split the remaining pair slots into single
 // tiles; the hardware hands CTAs out in index order, so the singles fill the SMs as the pairs finish.
 // Pair slot q = (group q % ng, token tiles 2 (q / ng) and 2 (q / ng) + 1).
-__global__ void __launch_bounds__(kMmaThreads, 1)
+__global__ void __launch_bounds__(kTileThreads, 1)
 ffn_gateup_tiles_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_g,
                         const __grid_constant__ CUtensorMap tm_u, const int32_t *__restrict__ glist, int ng, int n_pair,
                         int mtiles, int M, int d, int act_ld, __nv_bfloat16 *__restrict__ act, DeviceStatus *status) {
@@ -391,13 +395,15 @@ ffn_gateup_tiles_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_c
     } else {
         const int qd = warp & 3;                   // TMEM lane quarter this warp may read
         const int row = qd * 32 + lane;
+        const int slice = (warp - 2) >> 2, nslice = ((int)(blockDim.x >> 5) - 2) >> 2;
         if (mbar_wait(&bars->acc_ready, 0, bars, status)) {
             tc_fence_after();
-            for (int tt = 0; tt < ntile; ++tt) {
+#pragma unroll 1
+            for (int e = slice; e < ntile * 4; e += nslice) {   // chunk e: token tile e / 4, 32 channels e % 4
+                const int tt = e >> 2, cc = e & 3;
                 const int m = (mt0 + tt) * BM + row;
                 const uint32_t tbase = bars->tmem_base + ((uint32_t)(qd * 32) << 16) + (uint32_t)(tt * 256);
-#pragma unroll 1
-                for (int cc = 0; cc < 4; ++cc) {
+                {
                     uint32_t gv[32], uv[32];
                     tc_ld32(tbase + cc * 32, gv);
                     tc_ld32(tbase + 128 + cc * 32, uv);
@@ -426,7 +432,7 @@ ffn_gateup_tiles_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_c
 // ---- down -------------------------------------------------------------------------------------
 // grid (d / 256, token tiles, slices).  Slice z covers list entries [z*ng/Z, (z+1)*ng/Z).
 template <bool SPLIT>
-__global__ void __launch_bounds__(kMmaThreads, 1)
+__global__ void __launch_bounds__(kTileThreads, 1)
 ffn_down_mma_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant__ CUtensorMap tm_act_lo,
                     const __grid_constant__ CUtensorMap tm_wd, const int32_t *__restrict__ glist,
                     const int32_t *__restrict__ ng_dev, int ng_host, int M, int m_pad, int d,
@@ -461,16 +467,17 @@ ffn_down_mma_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_con
         if (lane == 0 && kblocks > 0) mma_loop<true, SPLIT>(t, kblocks, status);
     } else {
         const int q = warp & 3;
+        const int slice = (warp - 2) >> 2, nslice = ((int)(blockDim.x >> 5) - 2) >> 2;
         const int row = q * 32 + lane, m = mt * BM + row;
         float *dst = partial + ((size_t)z * m_pad + m) * d + (size_t)nt * BN;
         if (kblocks == 0) {   // empty slice: its partial is zero
-            if (m < M) for (int c = 0; c < BN; c += 4) *reinterpret_cast<float4 *>(dst + c) = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (m < M && slice == 0) for (int c = 0; c < BN; c += 4) *reinterpret_cast<float4 *>(dst + c) = make_float4(0.f, 0.f, 0.f, 0.f);
         } else if (mbar_wait(&t.bars->acc_ready, 0, t.bars, status)) {
             tc_fence_after();
             const uint32_t tbase = t.bars->tmem_base + ((uint32_t)(q * 32) << 16);
             const size_t o = (size_t)m * d + (size_t)nt * BN;      // one slice: the tile is the output itself
 #pragma unroll 1
-            for (int c = 0; c < BN / 32; ++c) {
+            for (int c = slice; c < BN / 32; c += nslice) {
                 uint32_t v[32];
                 tc_ld32(tbase + c * 32, v);
                 tc_wait_ld();
@@ -525,7 +532,7 @@ constexpr int BNW = 320;
 constexpr int kWideStage = kABytes + BNW * BK * 2;       // 16 KB + 40 KB
 constexpr int kWideStages = kRingBytesMma / kWideStage;  // 3
 
-__global__ void __launch_bounds__(kMmaThreads, 1)
+__global__ void __launch_bounds__(kTileThreads, 1)
 ffn_down_wide_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant__ CUtensorMap tm_wd,
                      const int32_t *__restrict__ glist, const int32_t *__restrict__ ng_dev, int ng_host, int M, int d,
                      const float *residual, float *out_f32, __nv_bfloat16 *__restrict__ out_bf16, DeviceStatus *status) {
@@ -576,13 +583,14 @@ ffn_down_wide_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_co
         }
     } else {
         const int q = warp & 3;
+        const int slice = (warp - 2) >> 2, nslice = ((int)(blockDim.x >> 5) - 2) >> 2;
         const int m = mt * BM + q * 32 + lane;
         if (kblocks > 0 && mbar_wait(&bars->acc_ready, 0, bars, status)) {
             tc_fence_after();
             const uint32_t tbase = bars->tmem_base + ((uint32_t)(q * 32) << 16);
             const size_t o = (size_t)m * d + (size_t)nt * BNW;
 #pragma unroll 1
-            for (int c = 0; c < BNW / 32; ++c) {
+            for (int c = slice; c < BNW / 32; c += nslice) {
                 uint32_t v[32];
                 tc_ld32(tbase + c * 32, v);
                 tc_wait_ld();
@@ -1201,14 +1209,14 @@ cs_status launch_ffn_mma(cs_plan *plan, const cs_layer *L, const void *X, const 
     {
         StageTimer timer(plan, CS_STAGE_EXEC, st);
         if (split)
-            ffn_gateup_mma_kernel<true><<<dim3(grid_g, mtiles), kMmaThreads, kMmaSmem, st>>>(
+            ffn_gateup_mma_kernel<true><<<dim3(grid_g, mtiles), kTileThreads, kMmaSmem, st>>>(
                 tm_x, tm_x_lo, tm_g, tm_u, glist, ng_dev, ng_host, M, c.d, act_ld, mask, act, act_lo, plan->status);
         else if (n_pair > 0) {
             // one shared support, its size known on the host: paired and single token tiles in one launch
-            ffn_gateup_tiles_kernel<<<dim3(n_pair + 2 * (slots - n_pair)), kMmaThreads, kMmaSmem, st>>>(
+            ffn_gateup_tiles_kernel<<<dim3(n_pair + 2 * (slots - n_pair)), kTileThreads, kMmaSmem, st>>>(
                 tm_x, tm_g, tm_u, glist, ng_host, n_pair, mtiles, M, c.d, act_ld, act, plan->status);
         } else
-            ffn_gateup_mma_kernel<false><<<dim3(grid_g, mtiles), kMmaThreads, kMmaSmem, st>>>(
+            ffn_gateup_mma_kernel<false><<<dim3(grid_g, mtiles), kTileThreads, kMmaSmem, st>>>(
                 tm_x, tm_x_lo, tm_g, tm_u, glist, ng_dev, ng_host, M, c.d, act_ld, mask, act, act_lo, plan->status);
         plan->launches++;
         CS_CUDA_TRY(plan, cudaGetLastError());
@@ -1221,14 +1229,14 @@ cs_status launch_ffn_mma(cs_plan *plan, const cs_layer *L, const void *X, const 
         const bool wide = !split && Z == 1 && c.d % BNW == 0 && ng_host > 0 &&
                           ((mtiles * (c.d / BNW) + sms - 1) / sms) * BNW < ((mtiles * ntiles + sms - 1) / sms) * BN;
         if (wide)
-            ffn_down_wide_kernel<<<dim3(c.d / BNW, mtiles), kMmaThreads, kMmaSmem, st>>>(
+            ffn_down_wide_kernel<<<dim3(c.d / BNW, mtiles), kTileThreads, kMmaSmem, st>>>(
                 tm_act, tm_wd, glist, ng_dev, ng_host, M, c.d, residual, out_f32, static_cast<__nv_bfloat16 *>(out_bf16), plan->status);
         else if (split)
-            ffn_down_mma_kernel<true><<<dim3(ntiles, mtiles, Z), kMmaThreads, kMmaSmem, st>>>(
+            ffn_down_mma_kernel<true><<<dim3(ntiles, mtiles, Z), kTileThreads, kMmaSmem, st>>>(
                 tm_act, tm_act_lo, tm_wd, glist, ng_dev, ng_host, M, m_pad, c.d, plan->mma_partial, residual, out_f32,
                 static_cast<__nv_bfloat16 *>(out_bf16), plan->status);
         else
-            ffn_down_mma_kernel<false><<<dim3(ntiles, mtiles, Z), kMmaThreads, kMmaSmem, st>>>(
+            ffn_down_mma_kernel<false><<<dim3(ntiles, mtiles, Z), kTileThreads, kMmaSmem, st>>>(
                 tm_act, tm_act_lo, tm_wd, glist, ng_dev, ng_host, M, m_pad, c.d, plan->mma_partial, residual, out_f32,
                 static_cast<__nv_bfloat16 *>(out_bf16), plan->status);
         plan->launches++;
