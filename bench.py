@@ -47,7 +47,6 @@ UNIT = "tokens/s"
 NCU_TRAFFIC = {
     ("l2_7b_b1", 22): 69.24e6 + 1.34e6,                       # ffn_gather_kernel
     ("l2_7b_b64", 22): 181.44e6 + 3.52e6 + 95.85e6 + 3.53e6,  # ffn_gateup_swap_kernel + ffn_down_swap_kernel
-    ("l2_13b_prompt", 27): 207.11e6 + 10.73e6 + 58.03e6 + 4.08e6,  # ffn_gateup_mma_kernel + ffn_down_wide_kernel
 }
 GRAPH_STEPS = 64          # most steps captured per CUDA graph
 N_TOKEN_BATCHES = 16      # distinct input batches rotated through
@@ -432,7 +431,7 @@ def bench_prompt(cfg, args, K, Wm, rank, world, local, dev, primary):
                 "d2h_bytes_per_step": cfg.B * cfg.d * 2},
         "gpu_launches": launches, "clocks": clocks.summary(),
         "region_ms": {"median": ms_region, "min": min(times), "max": max(times)},
-        "roofline": {"bound": "tensor", "kernel": "ffn_gateup_mma_kernel (ffn_gateup_tiles_kernel where paired token tiles shorten the last wave) + ffn_down_wide_kernel (ffn_down_mma_kernel where it needs fewer rounds)",
+        "roofline": {"bound": "tensor", "kernel": "ffn_gateup_tiles_kernel (paired token tiles where they shorten the last wave; else ffn_gateup_pair_kernel, CTA pairs with M = 256) + ffn_down_wide_kernel (ffn_down_mma_kernel where it needs fewer rounds)",
                      "achieved": achieved, "peak": tf_peak, "unit": "TFLOP/s", "frac": achieved / tf_peak,
                      "peak_kind": kind + " (sustained)", "flops_per_launch_pair": flops, "avg_pair_us": exec_us,
                      "duration_from": "cs_ffn_exec_shared on a given support, timed like the step (CUDA events, median of repeats)",

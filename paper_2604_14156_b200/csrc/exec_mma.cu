@@ -429,6 +429,154 @@ ffn_gateup_tiles_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_c
     teardown_cta(bars, warp, tcols);
 }
 
+// ---- gate / up for one shared support on CTA pairs (M = 256 across two SMs) ------------------------------
+// The single-CTA tiles above sit at shared-memory bandwidth: per 128 x 256 x 16 instruction the tensor pipe
+// reads 12 KB of operands while TMA refills the ring, 192 bytes per clock asked of a port that serves 128.
+// A pair of CTAs on neighbouring SMs (a cluster of two) issues ONE instruction of 256 token rows: each CTA
+// holds its own 128 token rows (A) and only HALF of the 256 weight columns (B: the even CTA the gate rows, the
+// odd CTA the up rows of the group), so a k block is 32 KB written and 32 KB read per CTA, which the port
+// can serve at the tensor pipe's full rate.  No multicast load: each CTA fetches its own tiles; its loads
+// signal the even CTA's barrier, whose MMA thread issues for both and frees both CTAs' slots with a
+// multicast commit.  grid = 2 x (ng x ceil(mtiles / 2)) CTAs in clusters of two; cluster q = (group q % ng,
+// token tiles 2 (q / ng) and 2 (q / ng) + 1).  A token tile beyond the batch is loaded as zeros and not stored.
+constexpr int kPairStageBytes = 2 * kABytes;                 // 16 KB of tokens + 16 KB of weights per CTA
+constexpr int kPairStages = kRingBytesMma / kPairStageBytes; // 6
+
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t saddr, uint32_t rank) {   // the same offset in CTA `rank`
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\nbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// TMA load of a CTA pair: data into this CTA's shared memory, bytes counted on a barrier given by its
+// cluster address (the even CTA's).
+__device__ __forceinline__ void tma_load_2d_pair(void *dst, const CUtensorMap *map, int x, int y, uint32_t bar_cluster) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(smem_u32(dst)), "l"(map), "r"(x), "r"(y), "r"(bar_cluster) : "memory");
+}
+__device__ __forceinline__ void tc_mma_pair(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n}"
+        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// Arrives (once the MMAs issued so far have completed) on the barrier at this offset in both CTAs of the pair.
+__device__ __forceinline__ void tc_commit_pair(uint64_t *bar) {
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(smem_u32(bar)), "h"((uint16_t)3) : "memory");
+}
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kTileThreads, 1)
+ffn_gateup_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_g,
+                       const __grid_constant__ CUtensorMap tm_u, const int32_t *__restrict__ glist, int ng, int M,
+                       int d, int act_ld, __nv_bfloat16 *__restrict__ act, DeviceStatus *status) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t rank = cluster_ctarank();                  // 0: gate half, issues the MMAs; 1: up half
+    const int q = blockIdx.x >> 1;
+    const int gi = q % ng, mt = 2 * (q / ng) + (int)rank;
+    const int g = glist[gi];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    uint8_t *base = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    Barriers *bars = reinterpret_cast<Barriers *>(base + kRingBytesMma);
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kMaxStages; ++s) { mbar_init(&bars->full[s], 1); mbar_init(&bars->empty[s], 1); }
+        mbar_init(&bars->acc_ready, 1);
+        bars->aborted = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {   // the same warp of both CTAs allocates for the pair
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(&bars->tmem_base)), "r"(256) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();        // the peer's barriers exist before anything signals them
+    tc_fence_after();
+    const int kblocks = d / BK;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            const uint32_t full0 = map_to_cta(smem_u32(&bars->full[0]), 0);   // the even CTA's full barriers
+            const CUtensorMap *tm_w = rank ? &tm_u : &tm_g;
+            int s = 0, ph = 1;
+            for (int kb = 0; kb < kblocks; ++kb, ++s) {
+                if (s == kPairStages) { s = 0; ph ^= 1; }
+                if (kb >= kPairStages && !mbar_wait(&bars->empty[s], ph, bars, status)) break;
+                uint8_t *st = base + (size_t)s * kPairStageBytes;
+                if (rank == 0) mbar_expect_tx(&bars->full[s], 2 * kPairStageBytes);   // both CTAs' bytes
+                tma_load_2d_pair(st, &tm_x, kb * BK, mt * BM, full0 + 8u * s);
+                tma_load_2d_pair(st + kABytes, tm_w, kb * BK, g * 128, full0 + 8u * s);
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0 && rank == 0) {
+            constexpr uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(256 >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
+            const uint32_t tmem = bars->tmem_base;
+            bool ok = true;
+            int s = 0, ph = 0;
+            for (int kb = 0; kb < kblocks && ok; ++kb, ++s) {
+                if (s == kPairStages) { s = 0; ph ^= 1; }
+                ok = mbar_wait(&bars->full[s], ph, bars, status);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t a0 = smem_u32(base + (size_t)s * kPairStageBytes), b0 = a0 + kABytes;
+#pragma unroll
+                for (int k4 = 0; k4 < BK / 16; ++k4)   // the descriptors' offsets hold in both CTAs' shared memory
+                    tc_mma_pair(tmem, desc_sw128(a0 + k4 * 32, 16), desc_sw128(b0 + k4 * 32, 16), idesc, (kb | k4) != 0);
+                tc_commit_pair(&bars->empty[s]);
+            }
+            if (ok) tc_commit_pair(&bars->acc_ready);
+        }
+    } else {
+        const int qd = warp & 3;
+        const int slice = (warp - 2) >> 2, nslice = ((int)(blockDim.x >> 5) - 2) >> 2;
+        const int m = mt * BM + qd * 32 + lane;
+        if (mbar_wait(&bars->acc_ready, 0, bars, status)) {
+            tc_fence_after();
+            const uint32_t tbase = bars->tmem_base + ((uint32_t)(qd * 32) << 16);
+#pragma unroll 1
+            for (int cc = slice; cc < 4; cc += nslice) {
+                uint32_t gv[32], uv[32];
+                tc_ld32(tbase + cc * 32, gv);
+                tc_ld32(tbase + 128 + cc * 32, uv);
+                tc_wait_ld();
+                uint32_t packed[16];
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                    const float a0 = silu_f(__uint_as_float(gv[2 * j])) * __uint_as_float(uv[2 * j]);
+                    const float a1 = silu_f(__uint_as_float(gv[2 * j + 1])) * __uint_as_float(uv[2 * j + 1]);
+                    const __nv_bfloat162 p = __floats2bfloat162_rn(a0, a1);
+                    packed[j] = *reinterpret_cast<const uint32_t *>(&p);
+                }
+                if (m < M) {
+                    uint4 *dst = reinterpret_cast<uint4 *>(act + (size_t)m * act_ld + (size_t)gi * 128 + cc * 32);
+#pragma unroll
+                    for (int j = 0; j < 4; ++j)
+                        dst[j] = make_uint4(packed[4 * j], packed[4 * j + 1], packed[4 * j + 2], packed[4 * j + 3]);
+                }
+            }
+        }
+    }
+    // Neither CTA leaves (or frees tensor memory) while the other may still read its shared memory or signal
+    // its barriers; every wait above is bounded, so both reach this point.
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(bars->tmem_base), "r"(256) : "memory");
+    }
+}
+
 // ---- down -------------------------------------------------------------------------------------
 // grid (d / 256, token tiles, slices).  Slice z covers list entries [z*ng/Z, (z+1)*ng/Z).
 template <bool SPLIT>
@@ -1154,6 +1302,7 @@ static int best_pair_count(int slots, int mtiles, int ng, int sms) {
 
 cs_status prepare_ffn_mma(cs_plan *plan) {
     CS_CUDA_TRY(plan, cudaFuncSetAttribute(ffn_gateup_tiles_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMmaSmem));
+    CS_CUDA_TRY(plan, cudaFuncSetAttribute(ffn_gateup_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMmaSmem));
     CS_CUDA_TRY(plan, cudaFuncSetAttribute(ffn_down_wide_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMmaSmem));
     CS_CUDA_TRY(plan, cudaFuncSetAttribute(ffn_gateup_mma_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMmaSmem));
     CS_CUDA_TRY(plan, cudaFuncSetAttribute(ffn_gateup_mma_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMmaSmem));
@@ -1199,7 +1348,8 @@ cs_status launch_ffn_mma(cs_plan *plan, const cs_layer *L, const void *X, const 
     // schedule of this shape, computed once); none leaves the launch to the single-tile kernel.
     int n_pair = 0;
     const int slots = ng_host * ((mtiles + 1) / 2);
-    if (!split && ng_dev == nullptr && mask == nullptr && ng_host > 0) {
+    const bool shared = !split && ng_dev == nullptr && mask == nullptr && ng_host > 0;
+    if (shared) {
         if (plan->pair_key_ng != ng_host || plan->pair_key_mtiles != mtiles) {
             plan->pair_count = best_pair_count(slots, mtiles, ng_host, plan->sm_count);
             plan->pair_key_ng = ng_host; plan->pair_key_mtiles = mtiles;
@@ -1211,7 +1361,13 @@ cs_status launch_ffn_mma(cs_plan *plan, const cs_layer *L, const void *X, const 
         if (split)
             ffn_gateup_mma_kernel<true><<<dim3(grid_g, mtiles), kTileThreads, kMmaSmem, st>>>(
                 tm_x, tm_x_lo, tm_g, tm_u, glist, ng_dev, ng_host, M, c.d, act_ld, mask, act, act_lo, plan->status);
-        else if (n_pair > 0) {
+        else if (shared && n_pair == 0) {
+            // one shared support and no gain from paired tiles (measured at k = 27 of 108 groups, 2048 tokens:
+            // 214 us for the GEMM pair against 223 us with single tiles; with paired tiles in play, k = 11 and
+            // 54, the mixed launch below is faster): CTA pairs, one M = 256 instruction over two token tiles
+            ffn_gateup_pair_kernel<<<dim3(2 * slots), kTileThreads, kMmaSmem, st>>>(
+                tm_x, tm_g, tm_u, glist, ng_host, M, c.d, act_ld, act, plan->status);
+        } else if (n_pair > 0) {
             // one shared support, its size known on the host: paired and single token tiles in one launch
             ffn_gateup_tiles_kernel<<<dim3(n_pair + 2 * (slots - n_pair)), kTileThreads, kMmaSmem, st>>>(
                 tm_x, tm_g, tm_u, glist, ng_host, n_pair, mtiles, M, c.d, act_ld, act, plan->status);
