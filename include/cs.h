@@ -357,6 +357,13 @@ int32_t cs_plan_crossover(const cs_plan *plan);
  * (CS_ERR_UNSUPPORTED otherwise).  On the shapes measured so far it is not faster than the plain chain
  * of launches (the recovery it overlaps costs less than the bookkeeping it adds), which is why it
  * is opt-in.
+ * on = 2 is the lighter form: the same single sketch-and-recovery launch, but the plain gather kernel
+ * behind it, which before it waits for the final supports only asks L2 (bulk prefetch) for the weight
+ * blocks of the first iterate's groups.  A hint and nothing else: supports and outputs are those of the
+ * plain path bit for bit.  Measured at the 7B shape it is not faster either (the gather kernel already
+ * streams at the HBM rate between its first request and its last row, and gains 2.5 us from weights that
+ * are all in L2, which the embedded recovery's exposed prologue costs again).
+ * on outside {0, 1, 2}: CS_ERR_SHAPE.
  */
 cs_status cs_plan_set_speculative(cs_plan *plan, int32_t on);
 

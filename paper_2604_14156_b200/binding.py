@@ -174,8 +174,9 @@ class Plan:
     def set_crossover(self, tokens: int):
         self.check(self.lib.cs_plan_set_crossover(self.handle, int(tokens)), "cs_plan_set_crossover")
 
-    def set_speculative(self, on: bool = True):
-        """Small batches: start the gather FFN on the recovery's first iterate (see include/cs.h)."""
+    def set_speculative(self, on=True):
+        """Small batches, on the recovery's first iterate: 1 / True = start the gather FFN's weight stream,
+        2 = only warm L2 with its weight blocks, 0 = the plain chain (see include/cs.h)."""
         self.check(self.lib.cs_plan_set_speculative(self.handle, int(on)), "cs_plan_set_speculative")
 
     def enable_timing(self, on: bool = True):

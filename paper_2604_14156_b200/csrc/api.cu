@@ -393,6 +393,13 @@ cs_status cs_layer_step(cs_plan *plan, const cs_layer *layer, const float *x, in
         // Opt-in (cs_plan_set_speculative): sketch and recovery in one launch, and the gather FFN behind it
         // starts its weight stream on the first iterate while the other iterations run.  (Not while stages
         // are being timed: event records between the launches would serialise them.)
+        if (plan->speculative == 2) {
+            // L2 warm-up only: the plain gather kernel, which asks L2 for the first iterate's blocks before it
+            // waits for the final supports
+            s = launch_sketch_recover(plan, layer, x, B, plan->y_buf, norm ? plan->n_buf : nullptr, sup, z_out, resid_out, st);
+            if (s != CS_OK) return s;
+            return launch_ffn_gather(plan, layer, n, sup, B, layer->add_residual ? x : nullptr, x_out, false, st, plan->slot_table);
+        }
         s = launch_sketch_recover(plan, layer, x, B, plan->y_buf, norm ? plan->n_buf : nullptr, support_out, z_out, resid_out, st);
         if (s != CS_OK) return s;
         return launch_ffn_gather_spec(plan, layer, n, B, layer->add_residual ? x : nullptr, x_out, st);
@@ -547,7 +554,8 @@ int32_t cs_plan_crossover(const cs_plan *plan) { return plan != nullptr ? plan->
 cs_status cs_plan_set_speculative(cs_plan *plan, int32_t on) {
     if (plan == nullptr) return CS_ERR_NULL;
     if (on && !sketch_recover_ok(plan)) return CS_ERR_UNSUPPORTED;
-    plan->speculative = on != 0;
+    if (on < 0 || on > 2) return CS_ERR_SHAPE;
+    plan->speculative = on;
     return CS_OK;
 }
 

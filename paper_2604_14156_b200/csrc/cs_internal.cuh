@@ -59,7 +59,7 @@ struct cs_plan {
     void *x_bf16;        // [2][max_tokens, d] bf16 activations: rounded value, then remainder
     void *act;           // [2][max_tokens, d_ff] bf16 SwiGLU activations over the group list (value, remainder)
     float *mma_partial;  // [slices, padded tokens, d] f32 partial down projections
-    int speculative;     // small batches: start the weight stream on the recovery's first iterate (opt-in)
+    int speculative;     // small batches, on the recovery's first iterate: 1 = start the weight stream, 2 = warm L2 only
     int mma_ok;          // shape qualifies for the tensor-core path
     int mma_min_tokens;  // smallest decode batch that takes it
     int mma_slices;      // most list slices the down GEMM is split into
@@ -127,9 +127,12 @@ cs_status launch_omp(cs_plan *plan, const float *Phi, const float *y, int B, int
 // the structured sketch (srht.cu)
 cs_status launch_sketch_srht(cs_plan *plan, const uint32_t *sign_bits, const int32_t *rows, const float *h, int B, float *y,
                              cudaStream_t st);
-// check: validate the supports on the device (ascending, distinct, in range) inside the same launch
+// check: validate the supports on the device (ascending, distinct, in range) inside the same launch.
+// warm: slot tables of a recovery still running in the launch ahead (launch_sketch_recover); the kernel
+// asks L2 for the weight blocks they name before it waits for the final supports.
 cs_status launch_ffn_gather(cs_plan *plan, const cs_layer *layer, const float *h, const int32_t *support,
-                            int B, const float *residual, float *out, bool check, cudaStream_t st);
+                            int B, const float *residual, float *out, bool check, cudaStream_t st,
+                            const int32_t *warm = nullptr);
 // The small-batch step: sketch and recovery in one launch, whose programmatic trigger fires when the
 // first iterate's slot table is in memory; the gather FFN launched behind it starts on that table,
 // follows the table while the iteration runs, and settles on the final one.

@@ -79,7 +79,7 @@ template <typename WT, int CPT, bool FULL, bool SPEC>
 __global__ void __launch_bounds__(SPEC ? kSpecThreads : kGatherThreads, 1)
 ffn_gather_kernel(const WT *__restrict__ Wg, const WT *__restrict__ Wu, const WT *__restrict__ Wdt,
                   const float *__restrict__ h, const int32_t *__restrict__ support, int d, int lb, int k, int G,
-                  float *__restrict__ partial, DeviceStatus *status, int check) {
+                  float *__restrict__ partial, DeviceStatus *status, int check, const int32_t *__restrict__ warm) {
     constexpr int E = Chunk<WT>::kElems;
     constexpr int DR = kLaneSlots / CPT;               // down rows in flight per thread
     constexpr int kSegElems = kUnitChunks * 32 * E;    // elements of one row segment
@@ -132,7 +132,27 @@ ffn_gather_kernel(const WT *__restrict__ Wg, const WT *__restrict__ Wu, const WT
     const int chunks = d / E;                                       // chunks per row
     const int nseg = (chunks + kUnitChunks * 32 - 1) / (kUnitChunks * 32);
     const int nunits = nrows * nseg;
-    if constexpr (!SPEC) pdl_wait();   // supports and activations come from the kernels before
+    if constexpr (!SPEC) {
+        // L2 warm-up (launched behind the sketch-and-recovery kernel, which triggers on its FIRST iterate):
+        // before the wait for the final support, every CTA asks L2 for its share of the weight blocks of the
+        // groups in the first iterate's slot table — nine tenths of them are in the final support, and HBM
+        // streams them while the remaining iterations run.  Only a hint: whatever the table holds at this
+        // moment, nothing but the range check stands between it and the request, and the pass below reads
+        // the final support as always.
+        if (warm != nullptr && tid < 3 * k) {
+            const int mat = tid / k, j = tid - mat * k;
+            const size_t chunk = ((size_t)d << lb) * sizeof(WT);            // one group's rows are contiguous
+            const size_t seg = ((chunk / nx) + 127) & ~(size_t)127;         // this CTA's share of each block
+            const size_t off = (size_t)bx * seg;
+            const int g = ld_visible(warm + (size_t)t * kSlotTablePitch + j);
+            if ((unsigned)g < (unsigned)G && off < chunk) {
+                const char *src = reinterpret_cast<const char *>(mat == 0 ? Wg : mat == 1 ? Wu : Wdt) + (size_t)g * chunk + off;
+                const uint32_t bytes = (uint32_t)min(seg, chunk - off);
+                asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(bytes) : "memory");
+            }
+        }
+        pdl_wait();   // supports and activations come from the kernels before
+    }
 
     if constexpr (!SPEC) {
         if (tid < nrows) {
@@ -447,12 +467,12 @@ cs_status launch_check_support(cs_plan *plan, const int32_t *support, int B, cud
 template <typename WT, bool SPEC>
 static void launch_gather_kernel(dim3 grid, cudaStream_t st, int cpt, int chunks, const WT *Wg, const WT *Wu,
                                  const WT *Wd, const float *h, const int32_t *sup, int d, int b, int k, int G,
-                                 float *partial, DeviceStatus *status, int check) {
+                                 float *partial, DeviceStatus *status, int check, const int32_t *warm) {
     const bool full = chunks % kGatherThreads == 0 && (cpt == 1 || cpt == 2 || cpt == 4);
     const int lb = b == 64 ? 6 : 7;
 #define CS_GATHER_CASE(N, F)                                                                              \
     launch_pdl(true, ffn_gather_kernel<WT, N, F, SPEC>, grid, dim3(SPEC ? kSpecThreads : kGatherThreads), kRingBytes, st, \
-               Wg, Wu, Wd, h, sup, d, lb, k, G, partial, status, check)
+               Wg, Wu, Wd, h, sup, d, lb, k, G, partial, status, check, warm)
     if (cpt <= 1) { if (full) CS_GATHER_CASE(1, true); else CS_GATHER_CASE(1, false); }
     else if (cpt <= 2) { if (full) CS_GATHER_CASE(2, true); else CS_GATHER_CASE(2, false); }
     else { if (full) CS_GATHER_CASE(4, true); else CS_GATHER_CASE(4, false); }
@@ -469,7 +489,8 @@ static int gather_nx(int sm_count, int nb, int rows_total, int nx_max) {
 // per token is left to the CTA that runs it; otherwise the supports are given (`check`: validate them).
 template <typename WT>
 static cs_status gather_typed(cs_plan *plan, const cs_layer *L, const float *h, const int32_t *support,
-                              int B, const float *residual, float *out, int check, bool spec, cudaStream_t st) {
+                              int B, const float *residual, float *out, int check, bool spec, cudaStream_t st,
+                              const int32_t *warm = nullptr) {
     const cs_config &c = plan->cfg;
     constexpr int E = Chunk<WT>::kElems;
     const int rows_total = c.k * c.group;
@@ -485,10 +506,11 @@ static cs_status gather_typed(cs_plan *plan, const cs_layer *L, const float *h, 
             StageTimer timer(plan, CS_STAGE_EXEC, st);
             if (spec)
                 launch_gather_kernel<WT, true>(grid, st, cpt, c.d / E, Wg, Wu, Wd, hp, support + (size_t)t0 * kSlotTablePitch,
-                                               c.d, c.group, c.k, plan->G, plan->partial, plan->status, 0);
+                                               c.d, c.group, c.k, plan->G, plan->partial, plan->status, 0, nullptr);
             else
                 launch_gather_kernel<WT, false>(grid, st, cpt, c.d / E, Wg, Wu, Wd, hp, support + (size_t)t0 * c.k, c.d,
-                                                c.group, c.k, plan->G, plan->partial, plan->status, check);
+                                                c.group, c.k, plan->G, plan->partial, plan->status, check,
+                                                warm != nullptr ? warm + (size_t)t0 * kSlotTablePitch : nullptr);
         }
         plan->launches++;
         CS_CUDA_TRY(plan, cudaGetLastError());
@@ -532,10 +554,10 @@ cs_status prepare_ffn_gather(cs_plan *plan) {
 }
 
 cs_status launch_ffn_gather(cs_plan *plan, const cs_layer *layer, const float *h, const int32_t *support,
-                            int B, const float *residual, float *out, bool check, cudaStream_t st) {
+                            int B, const float *residual, float *out, bool check, cudaStream_t st, const int32_t *warm) {
     if (plan->cfg.w_dtype == CS_BF16)
-        return gather_typed<__nv_bfloat16>(plan, layer, h, support, B, residual, out, check, false, st);
-    return gather_typed<float>(plan, layer, h, support, B, residual, out, check, false, st);
+        return gather_typed<__nv_bfloat16>(plan, layer, h, support, B, residual, out, check, false, st, warm);
+    return gather_typed<float>(plan, layer, h, support, B, residual, out, check, false, st, warm);
 }
 
 // The gather FFN behind launch_sketch_recover: starts on the recovery's first slot table (plan->slot_table).
@@ -588,7 +610,7 @@ static cudaError_t static_launch(const cs_config &c, const cs_layer *L, const fl
              *Wd = static_cast<const WT *>(L->Wd_t);
     dim3 grid(nx, B);
     launch_gather_kernel<WT, false>(grid, st, cpt, c.d / E, Wg, Wu, Wd, h, support, c.d, c.group, c.k, c.d_ff / c.group,
-                                    partial, static_cast<DeviceStatus *>(nullptr), 0);
+                                    partial, static_cast<DeviceStatus *>(nullptr), 0, nullptr);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     dim3 rgrid((c.d / 4 + kReduceCols - 1) / kReduceCols, B);

@@ -389,6 +389,28 @@ def test_layer_step_speculative_start(name, B):
     spec.close(); plain.close()
 
 
+@pytest.mark.parametrize("name,B", [("tiny_f32", 4), ("l2_7b_b1", 1), ("l2_7b_b1", 3), ("l2_7b_b64", 4)])
+def test_layer_step_l2_warmup(name, B):
+    """Mode 2 of the small-batch option (sketch + recovery in one launch, the plain gather kernel behind it
+    asking L2 for the first iterate's weight blocks before it waits for the final supports): the hint changes
+    no result, so parity with the oracle holds and, where no near-tie is excused, supports and outputs are
+    those of the plain chain bit for bit; repeated on the same plan."""
+    cfg = W.CONFIGS[name].with_(B=B)
+    L = _layer(cfg)
+    warm, plain = make_plan(cfg), make_plan(cfg)
+    warm.set_speculative(2)
+    for batch in range(3):
+        tk = W.make_tokens(cfg, L.A, batch=batch, B=B)
+        rep, _, _ = compare_layer_step(cfg, L, warm, tk.h)
+        want, sup, _, _ = cs.cs_layer_step(plain, device_layer(plain, L), tk.h.to(DEV))
+        got, sup2, _, _ = cs.cs_layer_step(warm, device_layer(warm, L), tk.h.to(DEV))
+        torch.cuda.synchronize()
+        assert warm.device_status() == 0
+        if rep.excused == 0:
+            assert torch.equal(sup, sup2) and torch.equal(got, want), batch
+    warm.close(); plain.close()
+
+
 def test_layer_step_speculative_random_shapes():
     """Random small-batch shapes through the opt-in path against the oracle and the plain chain."""
     rs = np.random.default_rng(11)
