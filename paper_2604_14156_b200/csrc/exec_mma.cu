@@ -437,10 +437,12 @@ ffn_gateup_tiles_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_c
 // odd CTA the up rows of the group), so a k block is 32 KB written and 32 KB read per CTA, which the port
 // can serve at the tensor pipe's full rate.  No multicast load: each CTA fetches its own tiles; its loads
 // signal the even CTA's barrier, whose MMA thread issues for both and frees both CTAs' slots with a
-// multicast commit.  grid = 2 x (ng x ceil(mtiles / 2)) CTAs in clusters of two; cluster q = (group q % ng,
-// token tiles 2 (q / ng) and 2 (q / ng) + 1).  A token tile beyond the batch is loaded as zeros and not stored.
+// multicast commit.  Pair slot q = (group q % ng, token tiles 2 (q / ng) and 2 (q / ng) + 1); the launch is
+// persistent, at most one cluster per SM pair, each taking every nc-th slot.  A token tile beyond the batch is
+// loaded as zeros and not stored.
 constexpr int kPairStageBytes = 2 * kABytes;                 // 16 KB of tokens + 16 KB of weights per CTA
 constexpr int kPairStages = kRingBytesMma / kPairStageBytes; // 6
+static_assert(kPairStages + 2 <= kMaxStages, "the two accumulator barriers of each kind follow the ring's");
 
 __device__ __forceinline__ uint32_t cluster_ctarank() {
     uint32_t r;
@@ -474,27 +476,38 @@ __device__ __forceinline__ void tc_commit_pair(uint64_t *bar) {
                  ::"r"(smem_u32(bar)), "h"((uint16_t)3) : "memory");
 }
 
+// Remote arrive on a barrier of the pair's even CTA (cluster address).
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t bar_cluster) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar_cluster) : "memory");
+}
+
+// Persistent: the launch has at most one cluster per SM pair, and cluster c takes the pair slots c, c + nc, ...
+// The TMA ring runs on across slot boundaries, and the accumulators alternate between the two halves of the 512
+// tensor-memory columns, so the set-up, the first loads and the epilogue of a slot (8.4 us of a 36 us round
+// when every slot was a cluster of its own) overlap the main loop of the next.  An accumulator half is reused
+// two slots later, once all epilogue warps of BOTH CTAs have arrived on its `acc_empty` barrier in the even CTA.
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kTileThreads, 1)
 ffn_gateup_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_g,
-                       const __grid_constant__ CUtensorMap tm_u, const int32_t *__restrict__ glist, int ng, int M,
-                       int d, int act_ld, __nv_bfloat16 *__restrict__ act, DeviceStatus *status) {
+                       const __grid_constant__ CUtensorMap tm_u, const int32_t *__restrict__ glist, int ng, int slots,
+                       int M, int d, int act_ld, __nv_bfloat16 *__restrict__ act, DeviceStatus *status) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t rank = cluster_ctarank();                  // 0: gate half, issues the MMAs; 1: up half
-    const int q = blockIdx.x >> 1;
-    const int gi = q % ng, mt = 2 * (q / ng) + (int)rank;
-    const int g = glist[gi];
+    const int c0 = blockIdx.x >> 1, nc = gridDim.x >> 1;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int nepi = (int)(blockDim.x >> 5) - 2;              // epilogue warps of one CTA
     uint8_t *base = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     Barriers *bars = reinterpret_cast<Barriers *>(base + kRingBytesMma);
+    uint64_t *acc_full = &bars->full[kPairStages], *acc_empty = &bars->empty[kPairStages];   // two each
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kMaxStages; ++s) { mbar_init(&bars->full[s], 1); mbar_init(&bars->empty[s], 1); }
-        mbar_init(&bars->acc_ready, 1);
+        for (int s = 0; s < kPairStages; ++s) { mbar_init(&bars->full[s], 1); mbar_init(&bars->empty[s], 1); }
+        mbar_init(&acc_full[0], 1); mbar_init(&acc_full[1], 1);
+        mbar_init(&acc_empty[0], 2 * nepi); mbar_init(&acc_empty[1], 2 * nepi);
         bars->aborted = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {   // the same warp of both CTAs allocates for the pair
         asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
-                     ::"r"(smem_u32(&bars->tmem_base)), "r"(256) : "memory");
+                     ::"r"(smem_u32(&bars->tmem_base)), "r"(512) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
     }
     tc_fence_before();
@@ -507,42 +520,56 @@ ffn_gateup_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_co
         if (lane == 0) {
             const uint32_t full0 = map_to_cta(smem_u32(&bars->full[0]), 0);   // the even CTA's full barriers
             const CUtensorMap *tm_w = rank ? &tm_u : &tm_g;
-            int s = 0, ph = 1;
-            for (int kb = 0; kb < kblocks; ++kb, ++s) {
-                if (s == kPairStages) { s = 0; ph ^= 1; }
-                if (kb >= kPairStages && !mbar_wait(&bars->empty[s], ph, bars, status)) break;
-                uint8_t *st = base + (size_t)s * kPairStageBytes;
-                if (rank == 0) mbar_expect_tx(&bars->full[s], 2 * kPairStageBytes);   // both CTAs' bytes
-                tma_load_2d_pair(st, &tm_x, kb * BK, mt * BM, full0 + 8u * s);
-                tma_load_2d_pair(st + kABytes, tm_w, kb * BK, g * 128, full0 + 8u * s);
+            int s = 0, ph = 1, it = 0;
+            bool ok = true;
+            for (int q = c0; q < slots && ok; q += nc) {
+                const int g = glist[q % ng], mt = 2 * (q / ng) + (int)rank;
+                for (int kb = 0; kb < kblocks; ++kb, ++s, ++it) {
+                    if (s == kPairStages) { s = 0; ph ^= 1; }
+                    if (it >= kPairStages && !mbar_wait(&bars->empty[s], ph, bars, status)) { ok = false; break; }
+                    uint8_t *st = base + (size_t)s * kPairStageBytes;
+                    if (rank == 0) mbar_expect_tx(&bars->full[s], 2 * kPairStageBytes);   // both CTAs' bytes
+                    tma_load_2d_pair(st, &tm_x, kb * BK, mt * BM, full0 + 8u * s);
+                    tma_load_2d_pair(st + kABytes, tm_w, kb * BK, g * 128, full0 + 8u * s);
+                }
             }
         }
     } else if (warp == 1) {
         if (lane == 0 && rank == 0) {
             constexpr uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(256 >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
-            const uint32_t tmem = bars->tmem_base;
             bool ok = true;
-            int s = 0, ph = 0;
-            for (int kb = 0; kb < kblocks && ok; ++kb, ++s) {
-                if (s == kPairStages) { s = 0; ph ^= 1; }
-                ok = mbar_wait(&bars->full[s], ph, bars, status);
-                if (!ok) break;
-                tc_fence_after();
-                const uint32_t a0 = smem_u32(base + (size_t)s * kPairStageBytes), b0 = a0 + kABytes;
+            int s = 0, ph = 0, j = 0;
+            for (int q = c0; q < slots && ok; q += nc, ++j) {
+                const int a = j & 1;
+                // the epilogues of the slot before last have left this half
+                if (j >= 2) { ok = mbar_wait(&acc_empty[a], ((j >> 1) - 1) & 1, bars, status); if (!ok) break; tc_fence_after(); }
+                const uint32_t tmem = bars->tmem_base + (uint32_t)(a * 256);
+                for (int kb = 0; kb < kblocks; ++kb, ++s) {
+                    if (s == kPairStages) { s = 0; ph ^= 1; }
+                    ok = mbar_wait(&bars->full[s], ph, bars, status);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t a0 = smem_u32(base + (size_t)s * kPairStageBytes), b0 = a0 + kABytes;
 #pragma unroll
-                for (int k4 = 0; k4 < BK / 16; ++k4)   // the descriptors' offsets hold in both CTAs' shared memory
-                    tc_mma_pair(tmem, desc_sw128(a0 + k4 * 32, 16), desc_sw128(b0 + k4 * 32, 16), idesc, (kb | k4) != 0);
-                tc_commit_pair(&bars->empty[s]);
+                    for (int k4 = 0; k4 < BK / 16; ++k4)   // the descriptors' offsets hold in both CTAs' shared memory
+                        tc_mma_pair(tmem, desc_sw128(a0 + k4 * 32, 16), desc_sw128(b0 + k4 * 32, 16), idesc, (kb | k4) != 0);
+                    tc_commit_pair(&bars->empty[s]);
+                }
+                if (ok) tc_commit_pair(&acc_full[a]);
             }
-            if (ok) tc_commit_pair(&bars->acc_ready);
         }
     } else {
         const int qd = warp & 3;
-        const int slice = (warp - 2) >> 2, nslice = ((int)(blockDim.x >> 5) - 2) >> 2;
-        const int m = mt * BM + qd * 32 + lane;
-        if (mbar_wait(&bars->acc_ready, 0, bars, status)) {
+        const int slice = (warp - 2) >> 2, nslice = nepi >> 2;
+        const uint32_t empty0 = map_to_cta(smem_u32(&acc_empty[0]), 0);   // the even CTA's acc_empty barriers
+        int j = 0;
+        for (int q = c0; q < slots; q += nc, ++j) {
+            const int a = j & 1;
+            const int gi = q % ng, mt = 2 * (q / ng) + (int)rank;
+            const int m = mt * BM + qd * 32 + lane;
+            if (!mbar_wait(&acc_full[a], (j >> 1) & 1, bars, status)) break;
             tc_fence_after();
-            const uint32_t tbase = bars->tmem_base + ((uint32_t)(qd * 32) << 16);
+            const uint32_t tbase = bars->tmem_base + ((uint32_t)(qd * 32) << 16) + (uint32_t)(a * 256);
 #pragma unroll 1
             for (int cc = slice; cc < 4; cc += nslice) {
                 uint32_t gv[32], uv[32];
@@ -551,19 +578,23 @@ ffn_gateup_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_co
                 tc_wait_ld();
                 uint32_t packed[16];
 #pragma unroll
-                for (int j = 0; j < 16; ++j) {
-                    const float a0 = silu_f(__uint_as_float(gv[2 * j])) * __uint_as_float(uv[2 * j]);
-                    const float a1 = silu_f(__uint_as_float(gv[2 * j + 1])) * __uint_as_float(uv[2 * j + 1]);
+                for (int jj = 0; jj < 16; ++jj) {
+                    const float a0 = silu_f(__uint_as_float(gv[2 * jj])) * __uint_as_float(uv[2 * jj]);
+                    const float a1 = silu_f(__uint_as_float(gv[2 * jj + 1])) * __uint_as_float(uv[2 * jj + 1]);
                     const __nv_bfloat162 p = __floats2bfloat162_rn(a0, a1);
-                    packed[j] = *reinterpret_cast<const uint32_t *>(&p);
+                    packed[jj] = *reinterpret_cast<const uint32_t *>(&p);
                 }
                 if (m < M) {
                     uint4 *dst = reinterpret_cast<uint4 *>(act + (size_t)m * act_ld + (size_t)gi * 128 + cc * 32);
 #pragma unroll
-                    for (int j = 0; j < 4; ++j)
-                        dst[j] = make_uint4(packed[4 * j], packed[4 * j + 1], packed[4 * j + 2], packed[4 * j + 3]);
+                    for (int jj = 0; jj < 4; ++jj)
+                        dst[jj] = make_uint4(packed[4 * jj], packed[4 * jj + 1], packed[4 * jj + 2], packed[4 * jj + 3]);
                 }
             }
+            // this warp has taken what it needs from the half: one arrival per warp, of both CTAs, frees it
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(empty0 + 8u * a);
         }
     }
     // Neither CTA leaves (or frees tensor memory) while the other may still read its shared memory or signal
@@ -573,7 +604,7 @@ ffn_gateup_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_co
     cluster_sync_all();
     if (warp == 1) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(bars->tmem_base), "r"(256) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(bars->tmem_base), "r"(512) : "memory");
     }
 }
 
@@ -1365,8 +1396,8 @@ cs_status launch_ffn_mma(cs_plan *plan, const cs_layer *L, const void *X, const 
             // one shared support and no gain from paired tiles (measured at k = 27 of 108 groups, 2048 tokens:
             // 214 us for the GEMM pair against 223 us with single tiles; with paired tiles in play, k = 11 and
             // 54, the mixed launch below is faster): CTA pairs, one M = 256 instruction over two token tiles
-            ffn_gateup_pair_kernel<<<dim3(2 * slots), kTileThreads, kMmaSmem, st>>>(
-                tm_x, tm_g, tm_u, glist, ng_host, M, c.d, act_ld, act, plan->status);
+            ffn_gateup_pair_kernel<<<dim3(2 * min(slots, plan->sm_count / 2)), kTileThreads, kMmaSmem, st>>>(
+                tm_x, tm_g, tm_u, glist, ng_host, slots, M, c.d, act_ld, act, plan->status);
         } else if (n_pair > 0) {
             // one shared support, its size known on the host: paired and single token tiles in one launch
             ffn_gateup_tiles_kernel<<<dim3(n_pair + 2 * (slots - n_pair)), kTileThreads, kMmaSmem, st>>>(
