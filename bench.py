@@ -47,6 +47,7 @@ UNIT = "tokens/s"
 NCU_TRAFFIC = {
     ("l2_7b_b1", 22): 69.24e6 + 1.34e6,                       # ffn_gather_kernel
     ("l2_7b_b64", 22): 181.44e6 + 3.52e6 + 95.85e6 + 3.53e6,  # ffn_gateup_swap_kernel + ffn_down_swap_kernel
+    ("l2_13b_prompt", 27): 211.12e6 + 12.08e6 + 56.08e6 + 5.21e6,  # ffn_gateup_pair_kernel + ffn_down_wide_kernel
 }
 GRAPH_STEPS = 64          # most steps captured per CUDA graph
 N_TOKEN_BATCHES = 16      # distinct input batches rotated through
