@@ -606,6 +606,28 @@ def test_layer_step_around_the_crossover_batch(B):
     print(B, rep)
 
 
+def test_plan_crossover_setting_moves_a_batch_between_the_paths():
+    """cs_plan_set_crossover: the same 6-token batch through the gather path (crossover above it) and through
+    the tensor cores (crossover below it) gives the oracle's result either way and the same supports; the
+    default is max(2, min(16, ceil(1.15 G / k))) and values outside 1..129 are refused."""
+    cfg = W.CONFIGS["l2_7b_b64"].with_(B=6)
+    L = _layer(cfg)
+    tk = W.make_tokens(cfg, L.A, B=6)
+    lo, hi = make_plan(cfg, max_tokens=6), make_plan(cfg, max_tokens=6)
+    assert lo.crossover == max(2, min(16, -(-115 * cfg.G // (100 * cfg.k))))
+    lo.set_crossover(2); hi.set_crossover(129)
+    assert lo.crossover == 2 and hi.crossover == 129
+    for bad in (0, 130, -3):
+        with pytest.raises(Exception):
+            lo.set_crossover(bad)
+    rep_lo, _, out_lo = compare_layer_step(cfg, L, lo, tk.h)
+    rep_hi, _, out_hi = compare_layer_step(cfg, L, hi, tk.h)
+    if rep_lo.excused == 0 and rep_hi.excused == 0:
+        assert rel(out_lo.cpu().numpy(), out_hi.cpu().numpy()) <= 2e-5
+    assert lo.launches != hi.launches     # different chains of kernels ran
+    lo.close(); hi.close()
+
+
 def test_ffn_exec_tensor_path_skips_unused_groups():
     """A batch whose supports leave most groups unused: the union list is short and ragged."""
     cfg = W.CONFIGS["l2_7b_b64"].with_(B=20, k=3)
