@@ -499,6 +499,39 @@ def test_layer_step_in_place_and_without_aux_outputs():
     assert torch.equal(again, ref_out)  # deterministic: no atomics on the path
 
 
+def test_every_regime_is_deterministic():
+    """No atomics and fixed summation orders everywhere: the same call twice (on a plan that has run other
+    work in between) gives the same bits, in the gather regime, on the decode GEMMs, and in the prompt-level
+    kernels (single tiles, paired tiles, CTA pairs)."""
+    for name, B in (("l2_7b_b1", 1), ("l2_7b_b1", 3), ("l2_7b_b64", 64), ("l3_8b_stack", 32)):
+        cfg = W.CONFIGS[name].with_(B=B, n_layers=1)
+        L = _layer(cfg)
+        plan = make_plan(cfg)
+        lay = device_layer(plan, L)
+        x = W.make_tokens(cfg, L.A, B=B).h.to(DEV)
+        other = W.make_tokens(cfg, L.A, batch=3, B=B).h.to(DEV)
+        first = [t.clone() for t in cs.cs_layer_step(plan, lay, x)]
+        cs.cs_layer_step(plan, lay, other)
+        second = cs.cs_layer_step(plan, lay, x)
+        torch.cuda.synchronize()
+        for a, b in zip(first, second):
+            assert torch.equal(a, b), (name, B)
+        plan.close()
+    for k in W.PROMPT_K_SWEEP:
+        cfg = W.CONFIGS["l2_13b_prompt"].with_(k=k)
+        L = _layer(cfg)
+        plan = make_plan(cfg)
+        lay = device_layer(plan, L)
+        H = W.make_tokens(cfg, L.A).h.to(DEV).to(torch.bfloat16)
+        sup = torch.arange(0, 2 * k, 2, dtype=torch.int32, device=DEV)
+        first = cs.cs_ffn_exec_shared(plan, lay, H, sup).clone()
+        cs.cs_ffn_exec_shared(plan, lay, H.flip(0).contiguous(), sup)
+        second = cs.cs_ffn_exec_shared(plan, lay, H, sup)
+        torch.cuda.synchronize()
+        assert plan.device_status() == 0 and torch.equal(first, second), k
+        plan.close()
+
+
 def test_stack_parity_teacher_forced_and_chained():
     """32 Llama-3-8B-shaped layers, batch 32.
     (i) Teacher forcing: every layer is fed the oracle's input for that layer; supports and outputs
